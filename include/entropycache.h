@@ -1,0 +1,144 @@
+/*
+ * libentropycache -- C ABI of the cached denoising step of EntropyCache
+ * (training-free KV caching for diffusion language models) on NVIDIA B200 (sm_100a).
+ *
+ * Three operations make up the data-parallel hot path of one denoising step:
+ *
+ *   ec_kv_refresh    scatter the active rows' freshly projected K/V into the
+ *                    full-context KV cache, in place          (Section 4.2; Appendix A, partial branch)
+ *   ec_attend        refresh, then bidirectional attention in which only the
+ *                    active rows are queries and every cached position is a key
+ *                                                              (Appendix A: TransformerBlock(Q[M u R], K[I], V[I]))
+ *   ec_entropy_gate  per-row softmax statistics of the logits (argmax,
+ *                    confidence, Shannon entropy), maximum entropy over the
+ *                    newly decoded rows, comparison with tau   (Eq. 1; Algorithm 1)
+ *
+ * "Active rows" are the mask tokens of the current block/window plus the k most
+ * recently decoded tokens (M u R); on a recompute step every row is active.
+ *
+ * General rules
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; the library
+ *     never allocates or frees device memory and keeps no pointer after a call
+ *     returns.  Descriptors (ec_attn_desc) are HOST structures, read during the call.
+ *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*;
+ *     NULL is the legacy default stream) and returns without synchronising.
+ *   - Tensors are dense and contiguous in the layouts given below.  Every base
+ *     pointer and every row (head_dim elements; a logits row) must start on a
+ *     16-byte boundary.
+ *   - The return value reports what the host can detect (null pointers, shapes,
+ *     alignment, workspace size, launch failure).  Conditions only the device can
+ *     see (a bounded wait that ran out) are written to the optional `dev_status`
+ *     word; kernels never trap.
+ *   - A workspace must be zero-filled once before its first use (ec_workspace_init
+ *     or any memset); calls leave it ready for the next call.  Two calls that may
+ *     overlap on the GPU need separate workspaces.
+ */
+#ifndef ENTROPYCACHE_H_
+#define ENTROPYCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EC_OK = 0,
+    EC_ERR_NULL = 1,        /* a required pointer is NULL */
+    EC_ERR_SHAPE = 2,       /* a size is non-positive, inconsistent or out of range */
+    EC_ERR_DTYPE = 3,       /* unknown ec_dtype */
+    EC_ERR_ALIGN = 4,       /* a base pointer or row is not 16-byte aligned */
+    EC_ERR_WORKSPACE = 5,   /* workspace missing or smaller than *_workspace_bytes() */
+    EC_ERR_UNSUPPORTED = 6, /* valid request outside what the kernels implement */
+    EC_ERR_CUDA = 7,        /* a CUDA runtime call or launch failed */
+    EC_ERR_TIMEOUT = 8      /* (dev_status only) a bounded device-side wait gave up */
+} ec_status;
+
+typedef enum { EC_F32 = 0, EC_BF16 = 1 } ec_dtype;
+
+/* gate decisions (Algorithm 1: "E <= tau" reuses the cache, otherwise full recompute) */
+enum { EC_SKIP = 0, EC_RECOMPUTE = 1 };
+
+/* Geometry of one layer's attention (host structure). */
+typedef struct {
+    int32_t batch;       /* sequences, >= 1 */
+    int32_t ctx_len;     /* L: prompt + generation positions held in the cache */
+    int32_t n_q_heads;   /* H_q */
+    int32_t n_kv_heads;  /* H_kv; H_q % H_kv == 0; query head h reads kv head h / (H_q/H_kv) */
+    int32_t head_dim;    /* D: 64 or 128 */
+    int32_t dtype;       /* ec_dtype of q, k_new, v_new, the caches and out */
+    float   scale;       /* softmax scale; 0 means 1/sqrt(head_dim) */
+} ec_attn_desc;
+
+/* Layouts
+ *   k_cache, v_cache  [batch, n_kv_heads, ctx_len, head_dim]
+ *   k_new, v_new      [batch, n_active,  n_kv_heads, head_dim]   (post-RoPE K)
+ *   q, out            [batch, n_active,  n_q_heads,  head_dim]   (post-RoPE Q)
+ *   active_idx        int32 [batch, n_active]; positions in [0, ctx_len), unique
+ *                     within a sequence (duplicates: the surviving row is
+ *                     unspecified).  NULL means the identity list 0..ctx_len-1
+ *                     and requires n_active == ctx_len (recompute step).
+ */
+
+/* Section 4.2 / Appendix A (partial branch): the active rows get fresh K,V, every
+ * other position keeps its cached K,V.
+ *     k_cache[b, h, active_idx[b,i], :] = k_new[b, i, h, :]     (same for V)
+ * Bytes are copied verbatim.  n_active == 0 is a no-op.  Indices outside
+ * [0, ctx_len) are skipped by the kernel (never written). */
+ec_status ec_kv_refresh(const ec_attn_desc *desc, void *k_cache, void *v_cache,
+                        const void *k_new, const void *v_new,
+                        const int32_t *active_idx, int32_t n_active, void *stream);
+
+/* Bytes of workspace ec_attend needs for this geometry and n_active (0 on bad arguments). */
+size_t ec_attend_workspace_bytes(const ec_attn_desc *desc, int32_t n_active);
+
+/* Appendix A, partial branch (and its full branch when n_active == ctx_len):
+ *   1. if k_new/v_new are given: refresh as ec_kv_refresh does;
+ *   2. out[b,i,hq,:] = sum_j softmax_j( scale * <q[b,i,hq,:], k_cache[b,hq/g,j,:]> ) * v_cache[b,hq/g,j,:]
+ *      over ALL j in [0, ctx_len), no mask (bidirectional attention), reading the
+ *      refreshed cache.  bf16 inputs: fp32 accumulation, bf16 output; fp32 inputs:
+ *      fp32 throughout.
+ * k_new and v_new may both be NULL to attend without refreshing.  workspace: at
+ * least ec_attend_workspace_bytes() bytes, 16-byte aligned, zero-filled before
+ * first use.  dev_status (nullable, device int32): set to an ec_status by the
+ * kernels if a bounded wait ran out; untouched otherwise. */
+ec_status ec_attend(const ec_attn_desc *desc, const void *q, const void *k_new, const void *v_new,
+                    void *k_cache, void *v_cache, const int32_t *active_idx, int32_t n_active,
+                    void *out, void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream);
+
+/* Bytes of workspace ec_entropy_gate needs (0 on bad arguments). */
+size_t ec_entropy_gate_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/* Eq. 1 and Algorithm 1.  For every logits row r (one pass over the row):
+ *     argmax_out[r]  = smallest j maximising logits[r, j]
+ *     conf_out[r]    = softmax(logits[r, :])[argmax]
+ *     entropy_out[r] = - sum_j p_j ln p_j          (nats; p = softmax of the row)
+ * and for every sequence b (rows b*rows_per_seq .. (b+1)*rows_per_seq - 1):
+ *     max_entropy_out[b] = max over rows with decoded_flags[r] != 0 of entropy (-inf if none)
+ *     decision_out[b]    = EC_RECOMPUTE if max_entropy_out[b] > tau else EC_SKIP
+ * logits: [n_rows, row_stride_elems] of `dtype`, only the first `vocab` columns of
+ * a row are read; -inf entries are allowed (probability 0), +inf/NaN are not.
+ * argmax_out / conf_out / entropy_out may each be NULL.  n_rows must be a
+ * multiple of rows_per_seq.  Arithmetic is fp32.  workspace as for ec_attend. */
+ec_status ec_entropy_gate(const void *logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                          int64_t row_stride_elems, int32_t rows_per_seq,
+                          const uint8_t *decoded_flags, float tau,
+                          int32_t *argmax_out, float *conf_out, float *entropy_out,
+                          float *max_entropy_out, int32_t *decision_out,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/* Zero-fills a workspace (asynchronous on `stream`). */
+ec_status ec_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/* Static, human-readable name of a status code. */
+const char *ec_status_string(int32_t status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int32_t ec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENTROPYCACHE_H_ */

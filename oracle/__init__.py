@@ -1,0 +1,150 @@
+"""CPU oracle for the EntropyCache hot path (fp64) -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes/numpy wrapper around ``ec_oracle.c``.  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import this package; the CUDA
+library and its Python binding never do, and this package imports neither of
+them.  Arrays are numpy arrays in storage encoding: float32, or uint16 holding
+bf16 bit patterns (dtype 0 / 1).
+
+Passages followed: Section 4.2 and Appendix A (partial step: refresh the active
+rows' K/V, attend from the active rows over every position), Eq. 1 and
+Algorithm 1 (entropy of each decoded row, maximum, comparison with tau).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ec_oracle.c")
+_SO = os.path.join(_HERE, "libec_oracle.so")
+_lib = None
+
+F32, BF16 = 0, 1
+SKIP, RECOMPUTE = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile ec_oracle.c with gcc (-O2, OpenMP) into libec_oracle.so beside it."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_SO)
+        vp, i32, i64, f64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double
+        lib.oracle_kv_refresh.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32]
+        lib.oracle_kv_refresh.restype = i32
+        lib.oracle_attend.argtypes = [i32, i32, i32, i32, i32, i32, f64, vp, vp, vp, i32, vp, i32, vp]
+        lib.oracle_attend.restype = i32
+        lib.oracle_entropy_gate.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float,
+                                            vp, vp, vp, vp, vp, vp]
+        lib.oracle_entropy_gate.restype = i32
+        lib.oracle_num_threads.restype = i32
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _storage(a: np.ndarray, dtype: int) -> np.ndarray:
+    want = np.float32 if dtype == F32 else np.uint16
+    if a.dtype != want or not a.flags.c_contiguous:
+        raise TypeError(f"expected contiguous {want.__name__} storage array, got {a.dtype}")
+    return a
+
+
+def kv_refresh(k_cache: np.ndarray, v_cache: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+               active_idx: np.ndarray | None, dtype: int) -> None:
+    """In place: cache[b, h, idx[b, i], :] <- new[b, i, h, :] (K and V).
+
+    k_cache/v_cache [B, H_kv, L, D]; k_new/v_new [B, n, H_kv, D]; active_idx
+    int32 [B, n] or None for the identity list 0..n-1 (recompute step)."""
+    for a in (k_cache, v_cache, k_new, v_new):
+        _storage(a, dtype)
+    B, Hkv, L, D = k_cache.shape
+    n = k_new.shape[1]
+    assert k_new.shape == (B, n, Hkv, D) and v_new.shape == k_new.shape and v_cache.shape == k_cache.shape
+    if active_idx is not None:
+        active_idx = np.ascontiguousarray(active_idx, dtype=np.int32)
+        assert active_idx.shape == (B, n)
+    rc = _load().oracle_kv_refresh(B, L, Hkv, D, k_cache.itemsize, _ptr(k_cache), _ptr(v_cache),
+                                   _ptr(k_new), _ptr(v_new), _ptr(active_idx), n)
+    if rc:
+        raise ValueError("oracle_kv_refresh: index out of range")
+
+
+def attend(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, dtype: int, *,
+           scale: float = 0.0, row_sel=None) -> np.ndarray:
+    """Bidirectional attention of the active rows over the whole cache.
+
+    q [B, n, H_q, D]; caches [B, H_kv, L, D] (already refreshed).  Returns
+    float64 [B, n_sel, H_q, D]; row_sel (list of indices into 0..n-1) restricts
+    the computed query rows, None computes all."""
+    for a in (q, k_cache, v_cache):
+        _storage(a, dtype)
+    B, n, Hq, D = q.shape
+    _, Hkv, L, _ = k_cache.shape
+    sel = None
+    rows = n
+    if row_sel is not None:
+        sel = np.ascontiguousarray(row_sel, dtype=np.int32)
+        rows = int(sel.size)
+    out = np.empty((B, rows, Hq, D), dtype=np.float64)
+    rc = _load().oracle_attend(B, L, Hq, Hkv, D, dtype, float(scale), _ptr(q), _ptr(k_cache),
+                               _ptr(v_cache), n, _ptr(sel), rows, _ptr(out))
+    if rc:
+        raise ValueError("oracle_attend: bad arguments")
+    return out
+
+
+def refresh_and_attend(q, k_new, v_new, k_cache, v_cache, active_idx, dtype, *, scale=0.0, row_sel=None):
+    """The layer-step as the paper orders it: refresh the active rows, then attend.
+    The caches are modified in place (pass copies to keep the pre-image)."""
+    if k_new is not None:
+        kv_refresh(k_cache, v_cache, k_new, v_new, active_idx, dtype)
+    return attend(q, k_cache, v_cache, dtype, scale=scale, row_sel=row_sel)
+
+
+def entropy_gate(logits: np.ndarray, dtype: int, vocab: int, decoded_flags: np.ndarray, tau: float,
+                 rows_per_seq: int | None = None, want_probs: bool = False) -> dict:
+    """Eq. 1 and the skip/recompute rule.
+
+    logits: storage array [R, row_stride] with row_stride >= vocab (only the
+    first `vocab` columns of each row are read).  Returns dict with argmax
+    int32[R], conf f64[R], entropy f64[R] (nats), max_entropy f64[B],
+    decision int32[B] (1 = recompute: E > tau; 0 = skip), probs (optional)."""
+    _storage(logits, dtype)
+    R, stride = logits.shape
+    assert stride >= vocab
+    rps = R if rows_per_seq is None else rows_per_seq
+    flags = np.ascontiguousarray(decoded_flags, dtype=np.uint8)
+    assert flags.shape == (R,)
+    nseq = R // rps if rps else 0
+    argmax = np.empty(R, np.int32)
+    conf = np.empty(R, np.float64)
+    ent = np.empty(R, np.float64)
+    maxh = np.empty(nseq, np.float64)
+    dec = np.empty(nseq, np.int32)
+    probs = np.empty((R, vocab), np.float64) if want_probs else None
+    rc = _load().oracle_entropy_gate(_ptr(logits), dtype, R, vocab, stride, rps, _ptr(flags),
+                                     ctypes.c_float(tau), _ptr(argmax), _ptr(conf), _ptr(ent),
+                                     _ptr(maxh), _ptr(dec), _ptr(probs))
+    if rc:
+        raise ValueError("oracle_entropy_gate: n_rows must be a multiple of rows_per_seq")
+    return dict(argmax=argmax, conf=conf, entropy=ent, max_entropy=maxh, decision=dec, probs=probs)
