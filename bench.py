@@ -1,0 +1,472 @@
+#!/usr/bin/env python
+"""Benchmark of the EntropyCache cached denoising step on B200 (libentropycache).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One *step* is one denoising step of the hot path over one batch of synthetic
+input: for every layer `ec_attend` (scatter-refresh of the active rows' K/V, then
+active-row bidirectional attention over the whole cache) followed by one
+`ec_entropy_gate` over the block's logits.  The headline `value` is the time of
+a SKIP step per layer (microseconds per layer-step: refresh + 34-row attention,
+plus the gate amortised over the layers); the same quantity for a RECOMPUTE step
+(every row active) is reported beside it, as the metric asks ("skip vs
+recompute").  Layers use distinct K/V caches whose total size exceeds the L2
+cache several times, so every layer-step streams its cache from HBM.
+
+Timing: CUDA events on the launching stream around exactly K replays of a CUDA
+graph that holds one whole step; W untimed warm-up replays first; max over ranks.
+With N > 1 every rank runs the same per-GPU workload on its own sequences (the
+path shards by sequence with no exchange): weak scaling, no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import ec_synth as syn  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+DEFAULT_WORKLOAD = "c2_llada_l768"
+
+
+def _peaks() -> dict:
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------- #
+# clocks sampler
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- #
+# device-side workload
+# --------------------------------------------------------------------------- #
+class DeviceWorkload:
+    """Synthetic tensors of one workload on one GPU: n_layers distinct K/V caches
+    (seeded torch generator on the device; same value laws as ec_synth)."""
+
+    def __init__(self, w: syn.Workload, n_layers: int, device, seed: int, need_recompute: bool = True):
+        import torch
+        import paper_2603_18489_b200 as ec
+
+        self.w, self.n_layers, self.ec, self.torch = w, n_layers, ec, torch
+        g = torch.Generator(device=device)
+        g.manual_seed(seed)
+        dt = torch.bfloat16 if w.dtype == syn.BF16 else torch.float32
+        B, L, Hq, Hkv, D = w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim
+        std = 1.0 / np.sqrt(D)
+
+        def rn(*shape):
+            return (torch.randn(*shape, generator=g, device=device, dtype=torch.float32) * std).to(dt)
+
+        self.desc = ec.make_desc(B, L, Hq, Hkv, D, w.dtype)
+        self.k_cache = [rn(B, Hkv, L, D) for _ in range(n_layers)]
+        self.v_cache = [rn(B, Hkv, L, D) for _ in range(n_layers)]
+        n = w.n_skip_rows
+        self.n_skip = n
+        self.q_s = [rn(B, n, Hq, D) for _ in range(n_layers)]
+        self.kn_s = [rn(B, n, Hkv, D) for _ in range(n_layers)]
+        self.vn_s = [rn(B, n, Hkv, D) for _ in range(n_layers)]
+        self.out_s = [torch.empty(B, n, Hq, D, device=device, dtype=dt) for _ in range(n_layers)]
+        idx = syn.active_rows(w, block_no=(w.gen_len // w.block) // 2)
+        self.idx_np = idx
+        self.idx = torch.from_numpy(idx).to(device)
+        self.ws_s = ec.new_workspace(ec.ec_attend_workspace_bytes(self.desc, n), device)
+        if need_recompute:
+            # one shared set of fresh tensors for the recompute step (every row active); each
+            # layer still owns its K/V cache, which is what the step streams and rewrites
+            self.q_r = rn(B, L, Hq, D)
+            self.kn_r = rn(B, L, Hkv, D)
+            self.vn_r = rn(B, L, Hkv, D)
+            self.out_r = torch.empty(B, L, Hq, D, device=device, dtype=dt)
+            self.ws_r = ec.new_workspace(ec.ec_attend_workspace_bytes(self.desc, L), device)
+        # logits: rows ~ N(0, sigma_r^2), sigma_r ~ U(0.5, 8); several buffers so a gate-only loop is cold
+        R = w.n_logit_rows
+        self.R = R
+        n_lbuf = max(2, int(np.ceil(2.2 * L2_BYTES / (R * w.vocab * syn.elem_bytes(w.dtype)))))
+        self.n_lbuf = min(n_lbuf, 40)
+        self.logits = []
+        for _ in range(self.n_lbuf):
+            sig = torch.rand(R, 1, generator=g, device=device) * 7.5 + 0.5
+            self.logits.append((torch.randn(R, w.vocab, generator=g, device=device) * sig).to(dt))
+        fl = syn.decoded_flags(R, 16, w.block, cfg_id=w.cfg_id)
+        self.flags_np = fl
+        self.flags = torch.from_numpy(fl).to(device)
+        self.ws_g = ec.new_workspace(ec.ec_entropy_gate_workspace_bytes(R, w.vocab), device)
+        nseq = R // w.block
+        self.maxh = torch.empty(nseq, device=device, dtype=torch.float32)
+        self.dec = torch.empty(nseq, device=device, dtype=torch.int32)
+        self.argmax = torch.empty(R, device=device, dtype=torch.int32)
+        self.conf = torch.empty(R, device=device, dtype=torch.float32)
+        self.ent = torch.empty(R, device=device, dtype=torch.float32)
+        self.tau = 1.5
+        self._gate_i = 0
+
+    # -- single calls (asynchronous on the current stream) ------------------------
+    def attend_skip(self, l: int, refresh: bool = True):
+        self.ec.ec_attend(self.desc, self.q_s[l], self.kn_s[l] if refresh else None,
+                          self.vn_s[l] if refresh else None, self.k_cache[l], self.v_cache[l], self.idx,
+                          out=self.out_s[l], workspace=self.ws_s)
+
+    def attend_recompute(self, l: int, refresh: bool = True):
+        self.ec.ec_attend(self.desc, self.q_r, self.kn_r if refresh else None, self.vn_r if refresh else None,
+                          self.k_cache[l], self.v_cache[l], None, out=self.out_r, workspace=self.ws_r)
+
+    def gate(self, i: int | None = None):
+        if i is None:
+            i = self._gate_i
+            self._gate_i = (self._gate_i + 1) % self.n_lbuf
+        self.ec.ec_entropy_gate(self.logits[i], self.w.vocab, self.w.block, self.flags, self.tau,
+                                argmax_out=self.argmax, conf_out=self.conf, entropy_out=self.ent,
+                                max_entropy_out=self.maxh, decision_out=self.dec, workspace=self.ws_g)
+
+    # -- algorithmic bytes / flops (per layer-step and per gate call) --------------
+    def skip_bytes(self) -> int:
+        w, s, n = self.w, syn.elem_bytes(self.w.dtype), self.n_skip
+        per_seq = (2 * w.ctx_len * w.n_kv_heads * w.head_dim * s + 4 * n * w.n_kv_heads * w.head_dim * s
+                   + 2 * n * w.n_q_heads * w.head_dim * s + 4 * n)
+        return per_seq * w.batch
+
+    def recompute_flops(self) -> int:
+        w = self.w
+        return 4 * w.ctx_len * w.ctx_len * w.head_dim * w.n_q_heads * w.batch
+
+    def gate_bytes(self) -> int:
+        return self.R * self.w.vocab * syn.elem_bytes(self.w.dtype) + 12 * self.R
+
+
+def _graph_time(torch, body, replays: int, warmup: int, stream) -> float:
+    """Captures body() into a CUDA graph, replays it `warmup` times untimed and `replays`
+    times timed; returns milliseconds per replay (CUDA events on the launching stream)."""
+    with torch.cuda.stream(stream):
+        body()  # eager once: first-call set-up (function attributes) must not happen under capture
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            body()
+        for _ in range(warmup):
+            g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(replays):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / replays
+
+
+def _choose_layers(w: syn.Workload) -> int:
+    per_layer = 2 * w.batch * w.ctx_len * w.n_kv_heads * w.head_dim * syn.elem_bytes(w.dtype)
+    need = int(np.ceil(3.0 * L2_BYTES / per_layer))
+    return int(min(max(need, 4), 64))
+
+
+# --------------------------------------------------------------------------- #
+# CPU oracle legs
+# --------------------------------------------------------------------------- #
+def _oracle_layer_step_us(w: syn.Workload, reps: int = 1) -> dict:
+    """Times the oracle (as it stands) on one skip layer-step and one gate call of workload w."""
+    import oracle
+
+    t = syn.attn_inputs(w, w.n_skip_rows)
+    lg = syn.logits_rows(w.n_logit_rows, w.vocab, w.dtype, cfg_id=w.cfg_id)
+    fl = syn.decoded_flags(w.n_logit_rows, 16, w.block, cfg_id=w.cfg_id)
+    oracle.entropy_gate(lg["logits"][:1], w.dtype, w.vocab, fl[:1], 1.5, 1)  # load + warm the library
+    ta, tg = [], []
+    for _ in range(reps):
+        kc, vc = t["k_cache"].copy(), t["v_cache"].copy()
+        t0 = time.perf_counter()
+        oracle.refresh_and_attend(t["q"], t["k_new"], t["v_new"], kc, vc, t["active_idx"], w.dtype)
+        t1 = time.perf_counter()
+        oracle.entropy_gate(lg["logits"], w.dtype, w.vocab, fl, 1.5, w.block)
+        t2 = time.perf_counter()
+        ta.append(t1 - t0)
+        tg.append(t2 - t1)
+    return dict(attend_us=min(ta) * 1e6, gate_us=min(tg) * 1e6, cores=oracle.num_threads())
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = syn.WORKLOADS[args.workload]
+    n_layers = _choose_layers(w)
+    for _ in range(args.warmup):
+        _oracle_layer_step_us(w, 1)
+    vals = []
+    cores = 1
+    for _ in range(args.steps):
+        r = _oracle_layer_step_us(w, 1)
+        cores = r["cores"]
+        vals.append(r["attend_us"] + r["gate_us"] / n_layers)
+    v = float(np.mean(vals))
+    sample = (f"per step: 1 skip layer-step (refresh + {w.n_skip_rows}-row attention over L={w.ctx_len}) "
+              f"+ 1 gate call [{w.n_logit_rows}x{w.vocab}] amortised over {n_layers} layers")
+    line = {
+        "impl": "reference", "metric": "us_per_layer_step_skip", "value": v, "unit": "us", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": v * n_layers / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "n_layers": n_layers, "l2": "n/a (host)"},
+        "cpu_baseline": {"value": v, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- #
+# main arm
+# --------------------------------------------------------------------------- #
+def run_cuda(args) -> None:
+    import torch
+    import paper_2603_18489_b200 as ec  # raises if the CUDA library is not built: no fallback
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+
+        dist = dist_
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = syn.WORKLOADS[args.workload]
+    n_layers = args.layers or _choose_layers(w)
+    peaks = _peaks()
+    wl = DeviceWorkload(w, n_layers, dev, seed=1234 + rank)
+    stream = torch.cuda.Stream(device=dev)
+    K, W = args.steps, max(args.warmup, 3)
+
+    def skip_step():
+        for l in range(n_layers):
+            wl.attend_skip(l)
+        wl.gate()
+
+    def recompute_step():
+        for l in range(n_layers):
+            wl.attend_recompute(l)
+        wl.gate()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def reduce_max(ms: float) -> float:
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- headline: K skip steps ----------------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    ms_skip = reduce_max(_graph_time(torch, skip_step, K, W, stream))
+    barrier()
+    ms_rec = reduce_max(_graph_time(torch, recompute_step, K, W, stream))
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- per-kernel regions for the rooflines (rank-local, same buffers, same stream) ----
+    def attend_only_skip():
+        for l in range(n_layers):
+            wl.attend_skip(l, refresh=False)
+
+    def attend_only_rec():
+        for l in range(n_layers):
+            wl.attend_recompute(l, refresh=False)
+
+    def gate_only():
+        for i in range(wl.n_lbuf):
+            wl.gate(i)
+
+    def refresh_only_skip():
+        for l in range(n_layers):
+            ec.ec_kv_refresh(wl.desc, wl.k_cache[l], wl.v_cache[l], wl.kn_s[l], wl.vn_s[l], wl.idx)
+
+    reps = max(K, 5)
+    ms_att_skip = _graph_time(torch, attend_only_skip, reps, 3, stream) / n_layers
+    ms_att_rec = _graph_time(torch, attend_only_rec, reps, 3, stream) / n_layers
+    ms_gate = _graph_time(torch, gate_only, reps, 3, stream) / wl.n_lbuf
+    ms_refresh = _graph_time(torch, refresh_only_skip, reps, 3, stream) / n_layers
+
+    # ---- end to end through the binding with host buffers --------------------------
+    dt = torch.bfloat16 if w.dtype == syn.BF16 else torch.float32
+    hq = [t.cpu().pin_memory() for t in wl.q_s]
+    hk = [t.cpu().pin_memory() for t in wl.kn_s]
+    hv = [t.cpu().pin_memory() for t in wl.vn_s]
+    hlog = wl.logits[0].cpu().pin_memory()
+    hout = [torch.empty_like(t, device="cpu").pin_memory() for t in wl.out_s]
+    hdec = torch.empty_like(wl.dec, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in hq + hk + hv) + hlog.numel() * hlog.element_size()
+    d2h = sum(t.numel() * t.element_size() for t in hout) + hdec.numel() * hdec.element_size()
+
+    def e2e_step():
+        with torch.cuda.stream(stream):
+            for l in range(n_layers):
+                wl.q_s[l].copy_(hq[l], non_blocking=True)
+                wl.kn_s[l].copy_(hk[l], non_blocking=True)
+                wl.vn_s[l].copy_(hv[l], non_blocking=True)
+                wl.attend_skip(l)
+                hout[l].copy_(wl.out_s[l], non_blocking=True)
+            wl.logits[0].copy_(hlog, non_blocking=True)
+            wl.gate(0)
+            hdec.copy_(wl.dec, non_blocking=True)
+        stream.synchronize()  # the host reads the decision to choose the next step's path
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(K):
+        e2e_step()
+    e1.record(stream)
+    stream.synchronize()
+    ms_e2e = reduce_max(e0.elapsed_time(e1) / K)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    us_skip = ms_skip * 1e3 / n_layers / world
+    us_rec = ms_rec * 1e3 / n_layers / world
+    skip_b, rec_f, gate_b = wl.skip_bytes(), wl.recompute_flops(), wl.gate_bytes()
+    att_gbs = skip_b / (ms_att_skip * 1e-3) / 1e9
+    rec_tf = rec_f / (ms_att_rec * 1e-3) / 1e12
+    gate_gbs = gate_b / (ms_gate * 1e-3) / 1e9
+
+    cpu = _oracle_layer_step_us(w, 2) if world == 1 or rank == 0 else None
+    n_split_kernels = 3  # refresh + attend + combine per skip layer-step
+    line = {
+        "metric": "us_per_layer_step_skip", "value": us_skip, "unit": "us", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms_skip, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.dtype == syn.BF16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "n_layers": n_layers, "batch": w.batch, "ctx_len": w.ctx_len,
+                   "n_active_skip": wl.n_skip, "vocab": w.vocab, "logit_rows": wl.R,
+                   "l2": f"inputs larger than L2: {n_layers} distinct K/V caches "
+                         f"({n_layers * 2 * w.batch * w.ctx_len * w.n_kv_heads * w.head_dim * syn.elem_bytes(w.dtype) >> 20} MiB) per step",
+                   "launch": "one CUDA graph per step"},
+        "recompute": {"us_per_layer_step": us_rec, "ms_per_step": ms_rec,
+                      "skip_over_recompute": us_skip / us_rec},
+        "kernels_us": {"attend_skip": ms_att_skip * 1e3, "attend_recompute": ms_att_rec * 1e3,
+                       "entropy_gate": ms_gate * 1e3, "kv_refresh_skip": ms_refresh * 1e3},
+        "roofline": {"kernel": "ec_attend skip path (attention + split merge)", "bound": "hbm",
+                     "achieved": att_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": att_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+        "roofline_recompute": {"kernel": "ec_attend recompute path", "bound": "tensor", "achieved": rec_tf,
+                               "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                               "frac": rec_tf / peaks["bf16_tflops"], "traffic": None,
+                               "peak_source": peaks["source"]},
+        "roofline_gate": {"kernel": "ec_entropy_gate", "bound": "hbm", "achieved": gate_gbs,
+                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gate_gbs / peaks["hbm_gbs"],
+                          "traffic": None, "peak_source": peaks["source"]},
+        "e2e": {"value": ms_e2e * 1e3 / n_layers / world, "unit": "us", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": K * (n_layers * n_split_kernels + 1),
+        "clocks": clocks,
+    }
+    if cpu is not None:
+        v = cpu["attend_us"] + cpu["gate_us"] / n_layers
+        line["cpu_baseline"] = {
+            "value": v, "unit": "us", "cores": cpu["cores"], "kind": "oracle",
+            "sample": f"1 skip layer-step ({wl.n_skip} rows over L={w.ctx_len}, {cpu['attend_us']:.0f} us) + 1 gate "
+                      f"call [{wl.R}x{w.vocab}] ({cpu['gate_us']:.0f} us) amortised over {n_layers} layers; best of 2"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(syn.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="distinct K/V caches per step (0: enough to exceed 3x L2)")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -160,7 +160,8 @@ def active_rows(w: Workload, block_no: int = 0, k_recent: int | None = None,
 def attn_inputs(w: Workload, n_active: int, *, step: int = 0, salt: int = 0,
                 std_qk: float | None = None, std_v: float | None = None,
                 identity_idx: bool | None = None, block_no: int = 0,
-                k_recent: int | None = None, shuffle_idx: bool = False) -> dict:
+                k_recent: int | None = None, shuffle_idx: bool = False,
+                active_idx: np.ndarray | None = None) -> dict:
     """Draws q, k_new, v_new (for the active rows) and the K/V caches.
 
     Layouts (all contiguous, storage dtype of the workload):
@@ -179,13 +180,16 @@ def attn_inputs(w: Workload, n_active: int, *, step: int = 0, salt: int = 0,
     sv = base if std_v is None else std_v
     B, L, Hq, Hkv = w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads
     if identity_idx is None:
-        identity_idx = (n_active == L)
+        identity_idx = (n_active == L) and active_idx is None
     q = _normal(_rng(w.cfg_id, T_Q, step, salt), (B, n_active, Hq, D), sqk)
     k_new = _normal(_rng(w.cfg_id, T_KNEW, step, salt), (B, n_active, Hkv, D), sqk)
     v_new = _normal(_rng(w.cfg_id, T_VNEW, step, salt), (B, n_active, Hkv, D), sv)
     k_cache = _normal(_rng(w.cfg_id, T_KCACHE, step, salt), (B, Hkv, L, D), sqk)
     v_cache = _normal(_rng(w.cfg_id, T_VCACHE, step, salt), (B, Hkv, L, D), sv)
-    if identity_idx:
+    if active_idx is not None:
+        idx = np.ascontiguousarray(active_idx, dtype=np.int32)
+        assert idx.shape == (B, n_active)
+    elif identity_idx:
         assert n_active == L
         idx = None
     else:

@@ -1,0 +1,195 @@
+"""Python binding of libentropycache (sm_100a CUDA kernels behind a C ABI).
+
+Argument marshalling only: every step of the hot path -- K/V refresh, active-row
+attention, the entropy gate -- runs in the library's kernels.  torch is used for
+device memory and streams.  There is no CPU fallback: importing this package
+without the built library raises.
+
+Functions carry the names of the C entry points declared in
+``include/entropycache.h``:
+
+    ec_kv_refresh(desc, k_cache, v_cache, k_new, v_new, active_idx)
+    ec_attend(desc, q, k_new, v_new, k_cache, v_cache, active_idx, ...)
+    ec_entropy_gate(logits, vocab, rows_per_seq, decoded_flags, tau, ...)
+
+(Section 4.2 / Appendix A / Eq. 1 and Algorithm 1 of the EntropyCache paper.)
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libentropycache.so")
+
+EC_F32, EC_BF16 = 0, 1
+EC_SKIP, EC_RECOMPUTE = 0, 1
+EC_OK = 0
+
+
+class EcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+class ec_attn_desc(ctypes.Structure):
+    """Mirror of the C struct ec_attn_desc."""
+    _fields_ = [("batch", ctypes.c_int32), ("ctx_len", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("scale", ctypes.c_float)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2603_18489_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    dp = ctypes.POINTER(ec_attn_desc)
+    lib.ec_kv_refresh.argtypes = [dp, vp, vp, vp, vp, vp, i32, vp]
+    lib.ec_kv_refresh.restype = i32
+    lib.ec_attend_workspace_bytes.argtypes = [dp, i32]
+    lib.ec_attend_workspace_bytes.restype = sz
+    lib.ec_attend.argtypes = [dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
+    lib.ec_attend.restype = i32
+    lib.ec_entropy_gate_workspace_bytes.argtypes = [i32, i32]
+    lib.ec_entropy_gate_workspace_bytes.restype = sz
+    lib.ec_entropy_gate.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.ec_entropy_gate.restype = i32
+    lib.ec_workspace_init.argtypes = [vp, sz, vp]
+    lib.ec_workspace_init.restype = i32
+    lib.ec_status_string.argtypes = [i32]
+    lib.ec_status_string.restype = ctypes.c_char_p
+    lib.ec_version.restype = i32
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.ec_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib.ec_version())
+
+
+def _check(status: int, where: str) -> None:
+    if status != EC_OK:
+        raise EcError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return EC_F32
+    if t.dtype == torch.bfloat16:
+        return EC_BF16
+    raise TypeError(f"unsupported element type {t.dtype}")
+
+
+def _dev(t: torch.Tensor | None, name: str):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no host path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def make_desc(batch: int, ctx_len: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype,
+              scale: float = 0.0) -> ec_attn_desc:
+    code = dtype if isinstance(dtype, int) else (EC_BF16 if dtype == torch.bfloat16 else EC_F32)
+    return ec_attn_desc(batch, ctx_len, n_q_heads, n_kv_heads, head_dim, code, scale)
+
+
+def desc_from_tensors(q: torch.Tensor, k_cache: torch.Tensor, scale: float = 0.0) -> ec_attn_desc:
+    B, _, Hq, D = q.shape
+    _, Hkv, L, _ = k_cache.shape
+    return make_desc(B, L, Hq, Hkv, D, _dtype_code(q), scale)
+
+
+def new_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
+    """Zero-filled device workspace of at least n_bytes (16-byte aligned by the allocator)."""
+    return torch.zeros(max(int(n_bytes), 16), dtype=torch.uint8, device=device)
+
+
+def ec_attend_workspace_bytes(desc: ec_attn_desc, n_active: int) -> int:
+    return int(lib.ec_attend_workspace_bytes(ctypes.byref(desc), int(n_active)))
+
+
+def ec_entropy_gate_workspace_bytes(n_rows: int, vocab: int) -> int:
+    return int(lib.ec_entropy_gate_workspace_bytes(int(n_rows), int(vocab)))
+
+
+def ec_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check(lib.ec_workspace_init(_dev(workspace, "workspace"), workspace.numel() * workspace.element_size(),
+                                 _stream(stream)), "ec_workspace_init")
+
+
+def ec_kv_refresh(desc: ec_attn_desc, k_cache, v_cache, k_new, v_new, active_idx, stream=None) -> None:
+    """k_cache[b, h, active_idx[b, i], :] = k_new[b, i, h, :] (and V), in place, asynchronously."""
+    n_active = int(k_new.shape[1])
+    _check(lib.ec_kv_refresh(ctypes.byref(desc), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"),
+                             _dev(k_new, "k_new"), _dev(v_new, "v_new"), _dev(active_idx, "active_idx"),
+                             n_active, _stream(stream)), "ec_kv_refresh")
+
+
+def ec_attend(desc: ec_attn_desc, q, k_new, v_new, k_cache, v_cache, active_idx, out=None,
+              workspace=None, dev_status=None, stream=None) -> torch.Tensor:
+    """Refresh the active rows (if k_new/v_new are given), then attend from the
+    active rows over the whole cache.  Returns `out` [B, n_active, H_q, D]."""
+    n_active = int(q.shape[1])
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(ec_attend_workspace_bytes(desc, n_active), q.device)
+    _check(lib.ec_attend(ctypes.byref(desc), _dev(q, "q"), _dev(k_new, "k_new"), _dev(v_new, "v_new"),
+                         _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"), _dev(active_idx, "active_idx"),
+                         n_active, _dev(out, "out"), _dev(workspace, "workspace"),
+                         workspace.numel() * workspace.element_size(), _dev(dev_status, "dev_status"),
+                         _stream(stream)), "ec_attend")
+    return out
+
+
+def ec_entropy_gate(logits, vocab: int, rows_per_seq: int, decoded_flags, tau: float, *,
+                    argmax_out=None, conf_out=None, entropy_out=None, max_entropy_out=None,
+                    decision_out=None, workspace=None, want_rows: bool = True, stream=None) -> dict:
+    """One pass over logits [R, row_stride]: per-row argmax / confidence / entropy,
+    per-sequence maximum entropy over the flagged rows and the skip (0) / recompute (1)
+    decision.  Outputs are device tensors; nothing is synchronised."""
+    if logits.dim() != 2 or not logits.is_cuda:
+        raise ValueError("logits must be a 2-D CUDA tensor [n_rows, row_stride]")
+    R, stride = int(logits.shape[0]), int(logits.stride(0))
+    dev = logits.device
+    n_seq = R // rows_per_seq if rows_per_seq > 0 else 0
+    if want_rows:
+        argmax_out = torch.empty(R, dtype=torch.int32, device=dev) if argmax_out is None else argmax_out
+        conf_out = torch.empty(R, dtype=torch.float32, device=dev) if conf_out is None else conf_out
+        entropy_out = torch.empty(R, dtype=torch.float32, device=dev) if entropy_out is None else entropy_out
+    if max_entropy_out is None:
+        max_entropy_out = torch.empty(n_seq, dtype=torch.float32, device=dev)
+    if decision_out is None:
+        decision_out = torch.empty(n_seq, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = new_workspace(ec_entropy_gate_workspace_bytes(R, vocab), dev)
+    if logits.stride(1) != 1:
+        raise ValueError("logits rows must be contiguous")
+    _check(lib.ec_entropy_gate(ctypes.c_void_p(logits.data_ptr()), _dtype_code(logits), R, int(vocab), stride,
+                               int(rows_per_seq), _dev(decoded_flags, "decoded_flags"), float(tau),
+                               _dev(argmax_out, "argmax_out"), _dev(conf_out, "conf_out"),
+                               _dev(entropy_out, "entropy_out"), _dev(max_entropy_out, "max_entropy_out"),
+                               _dev(decision_out, "decision_out"), _dev(workspace, "workspace"),
+                               workspace.numel() * workspace.element_size(), _stream(stream)), "ec_entropy_gate")
+    return dict(argmax=argmax_out, conf=conf_out, entropy=entropy_out, max_entropy=max_entropy_out,
+                decision=decision_out)

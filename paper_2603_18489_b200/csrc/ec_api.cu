@@ -1,0 +1,176 @@
+// C-ABI entry points of libentropycache: argument validation and dispatch.
+// Every check here is host-side; nothing in this file touches device memory.
+#include "ec_common.cuh"
+
+#include <atomic>
+
+namespace ec {
+
+int sm_count() {
+    static std::atomic<int> cached{0};
+    int v = cached.load(std::memory_order_relaxed);
+    if (v > 0) return v;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();  // no device (host-only use of the size queries): not sticky
+        return kDefaultSmCount;
+    }
+    cached.store(n, std::memory_order_relaxed);
+    return n;
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+ec_status check_desc(const ec_attn_desc* d) {
+    if (!d) return EC_ERR_NULL;
+    if (d->dtype != EC_F32 && d->dtype != EC_BF16) return EC_ERR_DTYPE;
+    if (d->batch < 1 || d->ctx_len < 1 || d->n_q_heads < 1 || d->n_kv_heads < 1) return EC_ERR_SHAPE;
+    if (d->n_q_heads % d->n_kv_heads != 0) return EC_ERR_SHAPE;
+    if (d->head_dim != 64 && d->head_dim != 128) return EC_ERR_UNSUPPORTED;
+    if (!(d->scale >= 0.f) || d->scale > 1.0e30f) return EC_ERR_SHAPE;  // also rejects NaN
+    return EC_OK;
+}
+
+ec_status check_active(const ec_attn_desc* d, const int32_t* active_idx, int32_t n_active) {
+    if (n_active < 0) return EC_ERR_SHAPE;
+    if (!active_idx && n_active != 0 && n_active != d->ctx_len) return EC_ERR_SHAPE;
+    if (active_idx && n_active > d->ctx_len) return EC_ERR_SHAPE;  // unique positions cannot exceed L
+    if (active_idx && (reinterpret_cast<uintptr_t>(active_idx) & 3u)) return EC_ERR_ALIGN;
+    return EC_OK;
+}
+
+}  // namespace
+}  // namespace ec
+
+using namespace ec;
+
+extern "C" {
+
+ec_status ec_kv_refresh(const ec_attn_desc* desc, void* k_cache, void* v_cache, const void* k_new,
+                        const void* v_new, const int32_t* active_idx, int32_t n_active, void* stream) {
+    ec_status st = check_desc(desc);
+    if (st != EC_OK) return st;
+    st = check_active(desc, active_idx, n_active);
+    if (st != EC_OK) return st;
+    if (n_active == 0) return EC_OK;
+    if (!k_cache || !v_cache || !k_new || !v_new) return EC_ERR_NULL;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_new) || !aligned16(v_new)) return EC_ERR_ALIGN;
+    const cudaError_t e =
+        launch_refresh(*desc, k_cache, v_cache, k_new, v_new, active_idx, n_active, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+size_t ec_attend_workspace_bytes(const ec_attn_desc* desc, int32_t n_active) {
+    if (check_desc(desc) != EC_OK || n_active < 0 || n_active > desc->ctx_len) return 0;
+    return attend_workspace_bytes(*desc, n_active);
+}
+
+ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, const void* v_new, void* k_cache,
+                    void* v_cache, const int32_t* active_idx, int32_t n_active, void* out, void* workspace,
+                    size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    ec_status st = check_desc(desc);
+    if (st != EC_OK) return st;
+    st = check_active(desc, active_idx, n_active);
+    if (st != EC_OK) return st;
+    if (n_active == 0) return EC_OK;
+    if (!q || !k_cache || !v_cache || !out) return EC_ERR_NULL;
+    if ((k_new == nullptr) != (v_new == nullptr)) return EC_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return EC_ERR_ALIGN;
+    if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return EC_ERR_ALIGN;
+    const size_t need = attend_workspace_bytes(*desc, n_active);
+    if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return EC_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    if (k_new) {
+        if (launch_refresh(*desc, k_cache, v_cache, k_new, v_new, active_idx, n_active, s) != cudaSuccess)
+            return EC_ERR_CUDA;
+    }
+    AttendArgs a;
+    a.d = *desc;
+    a.q = q;
+    a.k_cache = k_cache;
+    a.v_cache = v_cache;
+    a.n_active = n_active;
+    a.out = out;
+    a.workspace = workspace;
+    a.workspace_bytes = workspace_bytes;
+    a.dev_status = dev_status;
+    a.scale = desc->scale > 0.f ? desc->scale : 1.0f / sqrtf((float)desc->head_dim);
+    const cudaError_t e = desc->dtype == EC_BF16 ? launch_attend_bf16(a, s) : launch_attend_f32(a, s);
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+size_t ec_entropy_gate_workspace_bytes(int32_t n_rows, int32_t vocab) { return gate_workspace_bytes(n_rows, vocab); }
+
+ec_status ec_entropy_gate(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride_elems,
+                          int32_t rows_per_seq, const uint8_t* decoded_flags, float tau, int32_t* argmax_out,
+                          float* conf_out, float* entropy_out, float* max_entropy_out, int32_t* decision_out,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (dtype != EC_F32 && dtype != EC_BF16) return EC_ERR_DTYPE;
+    if (n_rows < 0 || vocab < 1 || rows_per_seq < 1 || row_stride_elems < vocab) return EC_ERR_SHAPE;
+    if (n_rows % rows_per_seq != 0) return EC_ERR_SHAPE;
+    if (n_rows > 65535) return EC_ERR_UNSUPPORTED;          // grid.y limit
+    if (vocab > 96 * 8192) return EC_ERR_UNSUPPORTED;       // split table of the workspace
+    if (tau != tau) return EC_ERR_SHAPE;
+    if (n_rows == 0) return EC_OK;
+    if (!logits || !decoded_flags || !max_entropy_out || !decision_out) return EC_ERR_NULL;
+    const size_t esize = dtype == EC_BF16 ? 2 : 4;
+    if (!aligned16(logits) || ((size_t)row_stride_elems * esize) % 16 != 0) return EC_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(argmax_out) | reinterpret_cast<uintptr_t>(conf_out) |
+         reinterpret_cast<uintptr_t>(entropy_out) | reinterpret_cast<uintptr_t>(max_entropy_out) |
+         reinterpret_cast<uintptr_t>(decision_out)) & 3u)
+        return EC_ERR_ALIGN;
+    const size_t need = gate_workspace_bytes(n_rows, vocab);
+    if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return EC_ERR_ALIGN;
+    GateArgs a;
+    a.logits = logits;
+    a.dtype = dtype;
+    a.n_rows = n_rows;
+    a.vocab = vocab;
+    a.row_stride = row_stride_elems;
+    a.rows_per_seq = rows_per_seq;
+    a.flags = decoded_flags;
+    a.tau = tau;
+    a.argmax_out = argmax_out;
+    a.conf_out = conf_out;
+    a.entropy_out = entropy_out;
+    a.max_entropy_out = max_entropy_out;
+    a.decision_out = decision_out;
+    a.workspace = workspace;
+    const cudaError_t e = launch_gate(a, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+ec_status ec_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (workspace_bytes == 0) return EC_OK;
+    if (!workspace) return EC_ERR_NULL;
+    return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? EC_OK
+               : EC_ERR_CUDA;
+}
+
+const char* ec_status_string(int32_t status) {
+    switch (status) {
+        case EC_OK: return "EC_OK";
+        case EC_ERR_NULL: return "EC_ERR_NULL: a required pointer is NULL";
+        case EC_ERR_SHAPE: return "EC_ERR_SHAPE: a size is non-positive, inconsistent or out of range";
+        case EC_ERR_DTYPE: return "EC_ERR_DTYPE: unknown element type";
+        case EC_ERR_ALIGN: return "EC_ERR_ALIGN: a pointer or row is not 16-byte aligned";
+        case EC_ERR_WORKSPACE: return "EC_ERR_WORKSPACE: workspace missing or too small";
+        case EC_ERR_UNSUPPORTED: return "EC_ERR_UNSUPPORTED: outside what the kernels implement";
+        case EC_ERR_CUDA: return "EC_ERR_CUDA: a CUDA runtime call or launch failed";
+        case EC_ERR_TIMEOUT: return "EC_ERR_TIMEOUT: a bounded device-side wait gave up";
+        default: return "unknown ec_status";
+    }
+}
+
+int32_t ec_version(void) { return 100; }
+
+}  // extern "C"

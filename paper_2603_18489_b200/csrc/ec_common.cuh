@@ -1,0 +1,73 @@
+// Shared declarations of libentropycache's CUDA translation units (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "entropycache.h"
+
+namespace ec {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Number of SMs the launch heuristics assume when the device cannot be queried
+// (B200: 148).
+constexpr int kDefaultSmCount = 148;
+
+int sm_count();  // cached cudaDevAttrMultiProcessorCount of the current device
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float fast_log2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---- internal launchers (host), one per translation unit ------------------
+struct GateArgs {
+    const void* logits;
+    int dtype;
+    int n_rows;
+    int vocab;
+    long long row_stride;
+    int rows_per_seq;
+    const uint8_t* flags;
+    float tau;
+    int* argmax_out;
+    float* conf_out;
+    float* entropy_out;
+    float* max_entropy_out;
+    int* decision_out;
+    void* workspace;
+};
+size_t gate_workspace_bytes(int n_rows, int vocab);
+cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream);
+
+cudaError_t launch_refresh(const ec_attn_desc& d, void* k_cache, void* v_cache, const void* k_new,
+                           const void* v_new, const int32_t* active_idx, int n_active,
+                           cudaStream_t stream);
+
+struct AttendArgs {
+    ec_attn_desc d;
+    const void* q;
+    const void* k_cache;
+    const void* v_cache;
+    int n_active;
+    void* out;
+    void* workspace;
+    size_t workspace_bytes;
+    int32_t* dev_status;
+    float scale;  // resolved (never 0)
+};
+size_t attend_workspace_bytes(const ec_attn_desc& d, int n_active);
+cudaError_t launch_attend_f32(const AttendArgs& a, cudaStream_t stream);
+cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);
+
+}  // namespace ec
