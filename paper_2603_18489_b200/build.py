@@ -1,6 +1,8 @@
 """Builds libentropycache.so (sm_100a only) in-tree, beside this file.
 
-    python -m paper_2603_18489_b200.build [--force] [--verbose]
+    python paper_2603_18489_b200/build.py [--force] [--verbose]
+
+(run by path: importing the package loads the library, which may not exist yet)
 
 Each .cu under csrc/ is compiled to an object under _build/ (git-ignored) and
 the objects are linked into one shared library with a static CUDA runtime, so
