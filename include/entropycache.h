@@ -129,6 +129,33 @@ ec_status ec_entropy_gate(const void *logits, int32_t dtype, int32_t n_rows, int
                           float *max_entropy_out, int32_t *decision_out,
                           void *workspace, size_t workspace_bytes, void *stream);
 
+/* Largest n_rows ec_entropy_gate_static accepts. */
+#define EC_GATE_STATIC_MAX_ROWS 256
+
+/* (The paper has no counterpart to this entry point: it is a packaging variant of
+ * ec_entropy_gate, not a step of the method.)
+ * ec_entropy_gate for callers that cannot allocate device memory and therefore have
+ * no workspace to pass: a serving process whose HBM is fully pre-partitioned, a
+ * plug-in that must not touch its host runtime's allocator, a step that cannot
+ * afford the device-wide synchronisation of cudaMalloc.  Same arguments, results
+ * and arithmetic as ec_entropy_gate, minus the workspace: the scratch is a
+ * fixed array inside the library image (about 390 KB, resident on every GPU that
+ * loads the library until the process exits).  The call allocates nothing.
+ *   - n_rows > EC_GATE_STATIC_MAX_ROWS returns EC_ERR_UNSUPPORTED (use
+ *     ec_entropy_gate with your own workspace); other argument errors as for
+ *     ec_entropy_gate.
+ *   - All calls on a GPU share the one scratch array: calls that may overlap on
+ *     the GPU race with each other; order them on one stream or with events.
+ *   - Each call clears the scratch words that must start at zero (an asynchronous
+ *     memset on `stream`), so a previous call's leftovers are harmless.
+ *   - The first call on each device resolves the scratch's device address; make
+ *     that first call outside any stream capture. */
+ec_status ec_entropy_gate_static(const void *logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                                 int64_t row_stride_elems, int32_t rows_per_seq,
+                                 const uint8_t *decoded_flags, float tau,
+                                 int32_t *argmax_out, float *conf_out, float *entropy_out,
+                                 float *max_entropy_out, int32_t *decision_out, void *stream);
+
 /* Zero-fills a workspace (asynchronous on `stream`). */
 ec_status ec_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 

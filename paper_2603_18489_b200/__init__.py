@@ -45,7 +45,7 @@ class ec_attn_desc(ctypes.Structure):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2603_18489_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2603_18489_b200/build.py` "
             "(there is no fallback path)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
@@ -60,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.ec_entropy_gate_workspace_bytes.restype = sz
     lib.ec_entropy_gate.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.ec_entropy_gate.restype = i32
+    lib.ec_entropy_gate_static.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
+    lib.ec_entropy_gate_static.restype = i32
     lib.ec_workspace_init.argtypes = [vp, sz, vp]
     lib.ec_workspace_init.restype = i32
     lib.ec_status_string.argtypes = [i32]
@@ -193,3 +195,26 @@ def ec_entropy_gate(logits, vocab: int, rows_per_seq: int, decoded_flags, tau: f
                                workspace.numel() * workspace.element_size(), _stream(stream)), "ec_entropy_gate")
     return dict(argmax=argmax_out, conf=conf_out, entropy=entropy_out, max_entropy=max_entropy_out,
                 decision=decision_out)
+
+
+EC_GATE_STATIC_MAX_ROWS = 256
+
+
+def ec_entropy_gate_static(logits, vocab: int, rows_per_seq: int, decoded_flags, tau: float, *,
+                           max_entropy_out, decision_out, argmax_out=None, conf_out=None, entropy_out=None,
+                           stream=None) -> None:
+    """ec_entropy_gate for callers that cannot allocate device memory (for example a
+    server whose HBM is fully pre-partitioned): the scratch is a fixed array inside the
+    library, so no workspace is passed and nothing is allocated -- which is also why every
+    output tensor must be supplied by the caller.  At most EC_GATE_STATIC_MAX_ROWS rows;
+    calls that may overlap on the GPU share the scratch and race; the first call on a
+    device should happen outside stream capture."""
+    if logits.dim() != 2 or not logits.is_cuda or logits.stride(1) != 1:
+        raise ValueError("logits must be a 2-D CUDA tensor with contiguous rows")
+    _check(lib.ec_entropy_gate_static(ctypes.c_void_p(logits.data_ptr()), _dtype_code(logits),
+                                      int(logits.shape[0]), int(vocab), int(logits.stride(0)), int(rows_per_seq),
+                                      _dev(decoded_flags, "decoded_flags"), float(tau),
+                                      _dev(argmax_out, "argmax_out"), _dev(conf_out, "conf_out"),
+                                      _dev(entropy_out, "entropy_out"), _dev(max_entropy_out, "max_entropy_out"),
+                                      _dev(decision_out, "decision_out"), _stream(stream)),
+           "ec_entropy_gate_static")
