@@ -3,6 +3,8 @@
 #include "ec_common.cuh"
 
 #include <atomic>
+#include <cstdlib>
+#include <cstring>
 
 namespace ec {
 
@@ -21,6 +23,25 @@ int sm_count() {
 }
 
 namespace {
+
+// bf16 with head_dim 128 runs on the tcgen05 kernel; everything else bf16 on the mma.sync kernel.
+// EC_ATTEND_IMPL=mma (environment, read once) forces the mma.sync kernel for A/B measurements.
+bool use_tc(const ec_attn_desc& d) {
+    static const bool forced_mma = [] {
+        const char* e = std::getenv("EC_ATTEND_IMPL");
+        return e && std::strcmp(e, "mma") == 0;
+    }();
+    return d.dtype == EC_BF16 && d.head_dim == 128 && !forced_mma;
+}
+
+size_t attend_ws(const ec_attn_desc& d, int n_active) {
+    size_t n = attend_workspace_bytes(d, n_active);
+    if (d.dtype == EC_BF16 && d.head_dim == 128) {
+        const size_t t = attend_tc_workspace_bytes(d, n_active);
+        if (t > n) n = t;
+    }
+    return n;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -65,7 +86,7 @@ ec_status ec_kv_refresh(const ec_attn_desc* desc, void* k_cache, void* v_cache, 
 
 size_t ec_attend_workspace_bytes(const ec_attn_desc* desc, int32_t n_active) {
     if (check_desc(desc) != EC_OK || n_active < 0 || n_active > desc->ctx_len) return 0;
-    return attend_workspace_bytes(*desc, n_active);
+    return attend_ws(*desc, n_active);
 }
 
 ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, const void* v_new, void* k_cache,
@@ -82,7 +103,7 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
         !aligned16(v_new))
         return EC_ERR_ALIGN;
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return EC_ERR_ALIGN;
-    const size_t need = attend_workspace_bytes(*desc, n_active);
+    const size_t need = attend_ws(*desc, n_active);
     if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
     if (!aligned16(workspace)) return EC_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -102,7 +123,9 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     a.workspace_bytes = workspace_bytes;
     a.dev_status = dev_status;
     a.scale = desc->scale > 0.f ? desc->scale : 1.0f / sqrtf((float)desc->head_dim);
-    const cudaError_t e = desc->dtype == EC_BF16 ? launch_attend_bf16(a, s) : launch_attend_f32(a, s);
+    const cudaError_t e = desc->dtype != EC_BF16 ? launch_attend_f32(a, s)
+                          : use_tc(*desc)        ? launch_attend_bf16_tc(a, s)
+                                                 : launch_attend_bf16(a, s);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 

@@ -68,6 +68,8 @@ struct AttendArgs {
 };
 size_t attend_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_f32(const AttendArgs& a, cudaStream_t stream);
-cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);
+cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);      // mma.sync path (any head_dim)
+size_t attend_tc_workspace_bytes(const ec_attn_desc& d, int n_active);
+cudaError_t launch_attend_bf16_tc(const AttendArgs& a, cudaStream_t stream);   // tcgen05 path (head_dim 128)
 
 }  // namespace ec

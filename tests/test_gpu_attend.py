@@ -21,9 +21,12 @@ def _gpu_attend(w, t, scale=0.0, refresh=True):
 
     d = ec.make_desc(w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, scale)
     gk, gv = to_dev(t["k_cache"]), to_dev(t["v_cache"])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
     out = ec.ec_attend(d, to_dev(t["q"]), to_dev(t["k_new"]) if refresh else None,
-                       to_dev(t["v_new"]) if refresh else None, gk, gv, to_dev(t["active_idx"]))
+                       to_dev(t["v_new"]) if refresh else None, gk, gv, to_dev(t["active_idx"]),
+                       dev_status=status)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0, f"device status {ec.status_string(int(status.item()))}"
     return out, gk, gv
 
 
