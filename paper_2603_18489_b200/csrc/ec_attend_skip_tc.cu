@@ -1,0 +1,663 @@
+// ec_attend, skip step (bf16, head_dim 128, at most 256 packed query rows per kv head):
+// ONE launch that refreshes the active rows' K/V in the cache, attends from the active
+// rows over the whole cache and merges the key-range partials -- no workspace, no second
+// kernel.  (Section 4.2 and Appendix A of the paper, partial branch:
+// TransformerBlock(Q[M u R], K[I], V[I]) after the rows M u R got fresh K, V.)
+//
+// The step is HBM-bound: every K/V byte of the cache is read exactly once.
+//   grid     (C, B*H_kv), launched as clusters of C CTAs: the C CTAs of a cluster share
+//            one (sequence, kv head) and split its 64-key tiles into C contiguous ranges;
+//   refresh  before its first load a CTA copies the fresh K/V rows whose positions fall
+//            in its own key range into the cache (no other CTA reads those rows), then
+//            orders the generic-proxy writes before its TMA reads;
+//   rows     the n_active x (H_q/H_kv) query rows that share the kv head are packed
+//            into one or two 128-row M tiles (NT); the same K/V tile serves both;
+//   pipeline warp 0 = TMA producer (K and V tiles [64 keys x 128] as two 64-column
+//            128-byte-swizzled boxes each, NS stages, full/empty mbarriers);
+//            warp 1 = tcgen05.mma issuer (S = Q K^T, M128 N64 K16 x 8, into one of two
+//            TMEM S buffers; O += P V, M128 N128 K16 x 4, P from shared memory, V
+//            MN-major); warps 2.. = softmax, thread = query row = TMEM lane (running
+//            max and sum, exp2 with the scale folded in, lazy rescale of O);
+//   merge    the CTAs of a cluster exchange their un-normalised (O, m, l) rows through
+//            distributed shared memory: row r goes to CTA r mod C, which combines the C
+//            partials, normalises and writes out[b, i, h, :].
+// Shared memory only holds the rows that exist: the tensor core always multiplies 128
+// rows, and the rows past the last packed query row read whatever follows in the CTA's
+// own allocation; rows of S, P and O are independent, so those values never reach a
+// real row and are never stored.
+// Every mbarrier wait is bounded: a wait that runs out sets EC_ERR_TIMEOUT in the
+// caller's dev_status word and a CTA-wide abort flag that makes all later waits fall
+// through; the CTA still takes part in the cluster barriers, frees its TMEM and exits.
+#include "ec_common.cuh"
+
+#include <cuda.h>
+
+namespace ec {
+namespace {
+
+constexpr int BM = 128, BN = 64, HD = 128;
+constexpr uint32_t KV_SUB = BN * 128;      // [64 keys x 64 bf16], 128-byte swizzle: 8 KB
+constexpr uint32_t KV_TILE = 2 * KV_SUB;   // [64 keys x 128 bf16]
+constexpr uint32_t STAGE = 2 * KV_TILE;    // K tile + V tile: 32 KB
+constexpr int kMaxStages = 6;
+constexpr int kRec = HD + 4;               // floats per exchanged row: O[128], m, l, pad (16-byte multiple)
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kMaxRows = 2 * BM;
+constexpr int kMaxCluster = 8;
+
+// barrier slots (8 bytes each)
+enum {
+    B_FULL = 0,                       // [kMaxStages]
+    B_EMPTY = kMaxStages,             // [kMaxStages]
+    B_SFULL = 2 * kMaxStages,         // [tile][2]
+    B_PFULL = B_SFULL + 4,            // [tile]
+    B_PVDONE = B_PFULL + 2,           // [tile]
+    B_COUNT = B_PVDONE + 2
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------
+__device__ __forceinline__ uint32_t s2u(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, parity)) return;
+        if ((i & 63) == 63 && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    if (dev_status) atomicExch(dev_status, (int)EC_ERR_TIMEOUT);
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// instruction descriptor: D fp32, A/B bf16, M = 128, N = n; b_mn = 1 when B is MN-major
+__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+struct SkipParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_new;   // nullptr: attend without refreshing
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    const int32_t* active_idx;    // nullptr: identity
+    __nv_bfloat16* out;
+    int32_t* dev_status;
+    int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
+    int n_splits, tiles_per_split, n_stages, rows_per_cta;
+    // shared-memory carve (bytes from the 1024-aligned base)
+    uint32_t off_q[2], off_p[2], rows_pad[2], off_stage, off_list, off_bar;
+    float scale_log2;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(64 + NT * 128, NT == 1 ? 2 : 1)
+attend_skip_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const SkipParams p) {
+    constexpr int kThreads = 64 + NT * 128;
+    constexpr uint32_t TM_COLS = NT * 256;   // per row tile: S0 [0,64), S1 [64,128), O [128,256)
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (s2u(smem_raw) + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - s2u(smem_raw));
+    const uint32_t bars = base + p.off_bar;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + p.off_bar + B_COUNT * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + p.off_bar + B_COUNT * 8 + 4);
+    int* list_count = reinterpret_cast<int*>(gbase + p.off_bar + B_COUNT * 8 + 8);
+    int2* list = reinterpret_cast<int2*>(gbase + p.off_list);   // (active row i, position) pairs of this CTA's key range
+    auto bar = [&](int idx) { return bars + idx * 8; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int split = blockIdx.x, bh = blockIdx.y;
+    const int b = bh / p.n_kv_heads, hk = bh % p.n_kv_heads;
+    const int n_tiles_total = (p.ctx_len + BN - 1) / BN;
+    const int t_begin = split * p.tiles_per_split;
+    const int t_end = min(n_tiles_total, t_begin + p.tiles_per_split);
+    const int T = t_end - t_begin;   // >= 1 by construction of the plan
+    const int NS = p.n_stages;
+
+    // ---- set-up: barriers, TMEM ----------------------------------------------------------
+    if (tid == 0) {
+        for (int i = 0; i < B_COUNT; ++i) {
+            uint32_t count = 1;
+            if (i >= B_PFULL && i < B_PFULL + 2) {
+                const int rows_t = min(BM, p.rows_total - (i - B_PFULL) * BM);
+                count = rows_t > 0 ? 32u * ((rows_t + 31) / 32) : 1u;
+            }
+            mbar_init(bar(i), count);
+        }
+        *abort_flag = 0;
+        *list_count = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(tmem_slot)), "r"(TM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+
+    // ---- refresh: fresh rows whose position lies in this CTA's key range ----------------------
+    const int key_lo = t_begin * BN, key_hi = min(p.ctx_len, t_end * BN);
+    if (p.k_new != nullptr) {
+        for (int i = tid; i < p.n_active; i += kThreads) {
+            const int pos = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
+            if (pos >= key_lo && pos < key_hi) list[atomicAdd(list_count, 1)] = make_int2(i, pos);
+        }
+    }
+    // Q rows of this kv head -> swizzled K-major tiles (rows past rows_total inside the padded tile are zero)
+    for (int t = 0; t < NT; ++t) {
+        const int rows_pad = (int)p.rows_pad[t];
+        for (int c = tid; c < rows_pad * (HD / 8); c += kThreads) {
+            const int row = c >> 4, ch = c & 15;
+            const int r = t * BM + row;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (r < p.rows_total) {
+                const int i = r / p.group, j = r % p.group;
+                v = __ldg(reinterpret_cast<const uint4*>(
+                    p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + j) * HD + ch * 8));
+            }
+            const uint32_t off = p.off_q[t] + (ch >> 3) * (uint32_t)rows_pad * 128u + (row >> 3) * 1024 + (row & 7) * 128 +
+                                 (((ch & 7) ^ (row & 7)) << 4);
+            *reinterpret_cast<uint4*>(gbase + off) = v;
+        }
+    }
+    __syncthreads();
+    const int n_mine = *list_count;
+    if (n_mine > 0) {   // block-uniform
+        for (int c = tid; c < n_mine * 32; c += kThreads) {
+            const int e = c >> 5, piece = c & 15, is_v = (c >> 4) & 1;
+            const int2 ip = list[e];
+            const long long src = (((long long)b * p.n_active + ip.x) * p.n_kv_heads + hk) * HD + piece * 8;
+            const long long dst = ((long long)bh * p.ctx_len + ip.y) * HD + piece * 8;
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src));
+            *reinterpret_cast<uint4*>((is_v ? p.v_cache : p.k_cache) + dst) = v;
+        }
+        __threadfence();
+        fence_async_global();   // generic-proxy writes above before this CTA's TMA reads of the same rows
+    }
+    fence_async_smem();         // Q tiles (generic proxy) -> visible to the tensor core (async proxy)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // softmax role: warp w >= 2 owns TMEM lanes 32 * (w % 4) of row tile (w - 2) / 4; thread = query row
+    const int soft_tile = warp >= 2 ? (warp - 2) >> 2 : 0;
+    const int soft_row = (warp & 3) * 32 + lane;
+    const int soft_rows_t = min(BM, p.rows_total - soft_tile * BM);
+    const bool soft_active = warp >= 2 && (warp & 3) * 32 < soft_rows_t;   // warp-uniform
+    const bool valid = soft_active && soft_row < soft_rows_t;
+    const uint32_t tm_t = tmem + ((uint32_t)((warp & 3) * 32) << 16) + soft_tile * 256;
+    float m_used = -INFINITY, l_run = 0.f;
+
+    if (warp == 0) {
+        // ================================ TMA producer ======================================
+        if (lane == 0) {
+            for (int j = 0; j < T; ++j) {
+                const int s = j % NS, u = j / NS;
+                const int key0 = (t_begin + j) * BN;
+                if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
+                const uint32_t dst = base + p.off_stage + s * STAGE;
+                mbar_expect_tx(bar(B_FULL + s), STAGE);
+                tma_load_3d(dst, &map_k, 0, key0, bh, bar(B_FULL + s));
+                tma_load_3d(dst + KV_SUB, &map_k, 64, key0, bh, bar(B_FULL + s));
+                tma_load_3d(dst + KV_TILE, &map_v, 0, key0, bh, bar(B_FULL + s));
+                tma_load_3d(dst + KV_TILE + KV_SUB, &map_v, 64, key0, bh, bar(B_FULL + s));
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ========================================
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = instr_desc(BN, 0), IDESC_PV = instr_desc(HD, 1);
+            auto issue_s = [&](int j) {
+                const uint32_t kst = base + p.off_stage + (j % NS) * STAGE;
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    const uint32_t d = tmem + t * 256 + (j & 1) * 64;
+                    const uint32_t qh = p.rows_pad[t] * 128u;   // bytes of one 64-column half of the Q tile
+#pragma unroll
+                    for (int k = 0; k < HD / 16; ++k) {
+                        tc_mma_ss(d, smem_desc(base + p.off_q[t] + (k >> 2) * qh + (k & 3) * 32, 16, 1024),
+                                  smem_desc(kst + (k >> 2) * KV_SUB + (k & 3) * 32, 16, 1024), IDESC_S, k > 0);
+                    }
+                    tc_commit(bar(B_SFULL + t * 2 + (j & 1)));
+                }
+            };
+            mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);
+            tc_fence_after();
+            issue_s(0);
+            for (int j = 0; j < T; ++j) {
+                if (j + 1 < T) {
+                    mbar_wait(bar(B_FULL + (j + 1) % NS), ((j + 1) / NS) & 1, abort_flag, p.dev_status);
+                    tc_fence_after();
+                    issue_s(j + 1);
+                }
+                const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + KV_TILE;
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    mbar_wait(bar(B_PFULL + t), j & 1, abort_flag, p.dev_status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < BN / 16; ++k) {
+                        tc_mma_ss(tmem + t * 256 + 128, smem_desc(base + p.off_p[t] + k * 32, 16, 1024),
+                                  smem_desc(vst + k * 2048, KV_SUB, 1024), IDESC_PV, (j > 0 || k > 0));
+                    }
+                    tc_commit(bar(B_PVDONE + t));
+                }
+                tc_commit(bar(B_EMPTY + j % NS));
+            }
+        }
+    } else if (soft_active) {
+        // ================================ softmax warps =====================================
+        const float sl2 = p.scale_log2;
+        unsigned char* prow = gbase + p.off_p[soft_tile] + (soft_row >> 3) * 1024 + (soft_row & 7) * 128;
+        const bool store_p = soft_row < (int)p.rows_pad[soft_tile];
+        const int t = soft_tile;
+
+        for (int j = 0; j < T; ++j) {
+            mbar_wait(bar(B_SFULL + t * 2 + (j & 1)), (j >> 1) & 1, abort_flag, p.dev_status);
+            tc_fence_after();
+            float sc[BN];
+            tc_ld32(tm_t + (j & 1) * 64, sc);
+            tc_ld32(tm_t + (j & 1) * 64 + 32, sc + 32);
+            tc_wait_ld();
+            const int key0 = (t_begin + j) * BN;
+            if (key0 + BN > p.ctx_len) {
+#pragma unroll
+                for (int c = 0; c < BN; ++c)
+                    if (key0 + c >= p.ctx_len) sc[c] = -INFINITY;
+            }
+            float mx = sc[0];
+#pragma unroll
+            for (int c = 1; c < BN; ++c) mx = fmaxf(mx, sc[c]);
+            if (!valid) mx = 0.f;                // padded lanes never ask for a rescale
+            const float m_tile = mx * sl2;
+            float factor = 1.f;
+            if (m_tile > m_used + 8.f || m_used == -INFINITY) {   // stale maximum allowed up to 2^8
+                factor = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_tile);
+                m_used = m_tile;
+            }
+            const bool need_rescale = (j > 0) && __any_sync(0xffffffffu, factor != 1.f);
+            float rs = 0.f;
+            const float mneg = -m_used;
+#pragma unroll
+            for (int c = 0; c < BN; ++c) {
+                sc[c] = fast_exp2(fmaf(sc[c], sl2, mneg));
+                rs += sc[c];
+            }
+            l_run = fmaf(l_run, factor, rs);
+
+            // P buffer free and O stable once P V of the previous tile has completed
+            if (j > 0) mbar_wait(bar(B_PVDONE + t), (j - 1) & 1, abort_flag, p.dev_status);
+            if (store_p) {   // rows past the padded tile have no storage
+#pragma unroll
+                for (int ch = 0; ch < BN / 8; ++ch) {
+                    uint4 v;
+                    v.x = pack2(sc[ch * 8 + 0], sc[ch * 8 + 1]);
+                    v.y = pack2(sc[ch * 8 + 2], sc[ch * 8 + 3]);
+                    v.z = pack2(sc[ch * 8 + 4], sc[ch * 8 + 5]);
+                    v.w = pack2(sc[ch * 8 + 6], sc[ch * 8 + 7]);
+                    *reinterpret_cast<uint4*>(prow + ((ch ^ (soft_row & 7)) << 4)) = v;
+                }
+            }
+            if (need_rescale) {
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < HD / 32; ++c) {
+                    float o[32];
+                    tc_ld32(tm_t + 128 + c * 32, o);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] *= factor;
+                    tc_st32(tm_t + 128 + c * 32, o);
+                }
+                tc_wait_st();
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(B_PFULL + t));
+        }
+        mbar_wait(bar(B_PVDONE + t), (T - 1) & 1, abort_flag, p.dev_status);
+        tc_fence_after();
+
+        if (p.n_splits == 1) {
+            // ---- single CTA per (sequence, kv head): normalise and store -----------------------
+            const int r = t * BM + soft_row;
+            const int i = valid ? r / p.group : 0, jh = valid ? r % p.group : 0;
+            __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD;
+            const float inv = 1.f / l_run;
+#pragma unroll
+            for (int c = 0; c < HD / 32; ++c) {
+                float o[32];
+                tc_ld32(tm_t + 128 + c * 32, o);
+                tc_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 w;
+                        w.x = pack2(o[v4 * 8 + 0] * inv, o[v4 * 8 + 1] * inv);
+                        w.y = pack2(o[v4 * 8 + 2] * inv, o[v4 * 8 + 3] * inv);
+                        w.z = pack2(o[v4 * 8 + 4] * inv, o[v4 * 8 + 5] * inv);
+                        w.w = pack2(o[v4 * 8 + 6] * inv, o[v4 * 8 + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
+                    }
+                }
+            }
+        }
+    }
+
+    if (p.n_splits > 1) {
+        // ---- merge across the cluster through distributed shared memory ----------------------
+        __syncwarp();
+        cluster_sync_all();   // every CTA of the cluster has left its main loop: staging memory is dead
+        if (soft_active) {
+            const int r = soft_tile * BM + soft_row;
+            const uint32_t owner = valid ? (uint32_t)(r % p.n_splits) : (uint32_t)split;
+            const uint32_t slot = valid ? (uint32_t)(split * p.rows_per_cta + r / p.n_splits) : 0u;
+            const uint32_t rec = map_to_cta(base + slot * (uint32_t)(kRec * 4), owner);
+#pragma unroll
+            for (int c = 0; c < HD / 32; ++c) {
+                float o[32];
+                tc_ld32(tm_t + 128 + c * 32, o);
+                tc_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 8; ++v4)
+                        st_cluster_f4(rec + (uint32_t)(c * 32 + v4 * 4) * 4u, o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2],
+                                      o[v4 * 4 + 3]);
+                }
+            }
+            if (valid) st_cluster_f4(rec + HD * 4u, m_used, l_run, 0.f, 0.f);
+        }
+        __syncwarp();
+        cluster_sync_all();   // every partial row has landed in its owner's shared memory
+        const float* recv = reinterpret_cast<const float*>(gbase);
+        const int n_own = (p.rows_total - split + p.n_splits - 1) / p.n_splits;   // rows r = split + q * C
+        for (int qi = warp; qi < n_own; qi += kThreads / 32) {
+            const int r = split + qi * p.n_splits;
+            float m = -INFINITY;
+            for (int s = 0; s < p.n_splits; ++s) m = fmaxf(m, recv[(s * p.rows_per_cta + qi) * kRec + HD]);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float l = 0.f;
+            for (int s = 0; s < p.n_splits; ++s) {
+                const float* rec = recv + (s * p.rows_per_cta + qi) * kRec;
+                const float w = fast_exp2(rec[HD] - m);
+                l = fmaf(w, rec[HD + 1], l);
+                const float4 o = *reinterpret_cast<const float4*>(rec + lane * 4);
+                acc.x = fmaf(w, o.x, acc.x);
+                acc.y = fmaf(w, o.y, acc.y);
+                acc.z = fmaf(w, o.z, acc.z);
+                acc.w = fmaf(w, o.w, acc.w);
+            }
+            const int i = r / p.group, jh = r % p.group;
+            __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD;
+            const float inv = 1.f / l;
+            uint2 w2;
+            w2.x = pack2(acc.x * inv, acc.y * inv);
+            w2.y = pack2(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(dst + lane * 4) = w2;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// cache [B*Hkv, L, 128] bf16 -> 3-D map {d, key, head}; box {64, 64, 1}; 128-byte swizzle; keys beyond L read as zero
+bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)ctx_len, (cuuint64_t)bh};
+    const cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)ctx_len * HD * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)BN, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(cache), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct SkipPlan {
+    int nt, rows_total, n_splits, tiles_per_split, n_stages, rows_per_cta;
+    uint32_t off_q[2], off_p[2], rows_pad[2], off_stage, off_list, off_bar, smem_bytes;
+};
+
+constexpr uint32_t kSmemTwoPerSm = 115712;   // (228 KB per SM - 2 x 1 KB reserved) / 2
+constexpr uint32_t kSmemMax = 232448;        // 227 KB: largest dynamic allocation of one CTA
+
+SkipPlan make_skip_plan(const ec_attn_desc& d, int n_active) {
+    SkipPlan pl{};
+    const int g = d.n_q_heads / d.n_kv_heads;
+    pl.rows_total = n_active * g;
+    pl.nt = pl.rows_total > BM ? 2 : 1;
+    const int key_tiles = (d.ctx_len + BN - 1) / BN;
+    const int bh = d.batch * d.n_kv_heads;
+    const int slots = (pl.nt == 1 ? 2 : 1) * sm_count();   // co-resident CTAs
+    int c = slots / bh;
+    if (c < 1) c = 1;
+    if (c > kMaxCluster) c = kMaxCluster;
+    if (c > key_tiles) c = key_tiles;
+    pl.tiles_per_split = (key_tiles + c - 1) / c;
+    pl.n_splits = (key_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
+    pl.rows_per_cta = (pl.rows_total + pl.n_splits - 1) / pl.n_splits;
+    uint32_t off = 0;
+    for (int t = 0; t < 2; ++t) {
+        const int rows_t = t < pl.nt ? (pl.rows_total - t * BM < BM ? pl.rows_total - t * BM : BM) : 0;
+        pl.rows_pad[t] = (uint32_t)((rows_t + 7) / 8 * 8);
+        pl.off_q[t] = off;
+        off += pl.rows_pad[t] * 256u;
+    }
+    for (int t = 0; t < 2; ++t) {
+        pl.off_p[t] = off;
+        off += pl.rows_pad[t] * 128u;
+    }
+    pl.off_stage = off;   // multiple of 1024: every piece above is a multiple of 8 rows x 128 bytes
+    const uint32_t tail = (uint32_t)n_active * 8u + 16u + B_COUNT * 8u + 16u + 1024u;   // list, barriers, alignment slack
+    int ns = 3;
+    if (off + 3 * STAGE + tail > kSmemTwoPerSm || pl.nt == 2) {
+        ns = (int)((kSmemMax - off - tail) / STAGE);
+        if (ns > kMaxStages) ns = kMaxStages;
+    }
+    if (ns > pl.tiles_per_split && pl.tiles_per_split >= 2) ns = pl.tiles_per_split;
+    if (ns < 2) ns = 2;
+    pl.n_stages = ns;
+    off += (uint32_t)ns * STAGE;
+    pl.off_list = off;
+    off += ((uint32_t)n_active * 8u + 15u) & ~15u;
+    pl.off_bar = off;
+    off += B_COUNT * 8u + 16u;
+    pl.smem_bytes = off + 1024u;
+    return pl;
+}
+
+template <int NT>
+cudaError_t launch_nt(const SkipPlan& pl, const SkipParams& p, const CUtensorMap& mk, const CUtensorMap& mv, int bh,
+                      cudaStream_t stream) {
+    static bool attr_done[64] = {};   // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        const cudaError_t e =
+            cudaFuncSetAttribute(attend_skip_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(pl.n_splits, bh, 1);
+    cfg.blockDim = dim3(64 + NT * 128, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = pl.n_splits;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attend_skip_kernel<NT>, mk, mv, p);
+}
+
+}  // namespace
+
+bool attend_skip_supported(const ec_attn_desc& d, int n_active) {
+    if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
+    const long long rows = (long long)n_active * (d.n_q_heads / d.n_kv_heads);
+    if (rows > kMaxRows) return false;
+    if ((long long)d.batch * d.n_kv_heads > 65535) return false;   // grid.y
+    const SkipPlan pl = make_skip_plan(d, n_active);
+    // the exchange buffer (C x rows_per_cta records) reuses the staging memory below the barrier block
+    const size_t recv = (size_t)pl.n_splits * pl.rows_per_cta * kRec * sizeof(float);
+    return pl.smem_bytes <= kSmemMax && pl.n_stages >= 2 && recv <= pl.off_list;
+}
+
+cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
+                               cudaStream_t stream) {
+    const SkipPlan pl = make_skip_plan(a.d, a.n_active);
+    const int bh = a.d.batch * a.d.n_kv_heads;
+    CUtensorMap map_k, map_v;
+    if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
+        return cudaErrorInvalidValue;
+    SkipParams p{};
+    p.q = static_cast<const __nv_bfloat16*>(a.q);
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.k_cache = static_cast<__nv_bfloat16*>(const_cast<void*>(a.k_cache));
+    p.v_cache = static_cast<__nv_bfloat16*>(const_cast<void*>(a.v_cache));
+    p.active_idx = active_idx;
+    p.out = static_cast<__nv_bfloat16*>(a.out);
+    p.dev_status = a.dev_status;
+    p.n_active = a.n_active;
+    p.ctx_len = a.d.ctx_len;
+    p.n_q_heads = a.d.n_q_heads;
+    p.n_kv_heads = a.d.n_kv_heads;
+    p.group = a.d.n_q_heads / a.d.n_kv_heads;
+    p.rows_total = pl.rows_total;
+    p.n_splits = pl.n_splits;
+    p.tiles_per_split = pl.tiles_per_split;
+    p.n_stages = pl.n_stages;
+    p.rows_per_cta = pl.rows_per_cta;
+    for (int t = 0; t < 2; ++t) {
+        p.off_q[t] = pl.off_q[t];
+        p.off_p[t] = pl.off_p[t];
+        p.rows_pad[t] = pl.rows_pad[t];
+    }
+    p.off_stage = pl.off_stage;
+    p.off_list = pl.off_list;
+    p.off_bar = pl.off_bar;
+    p.scale_log2 = a.scale * kLog2e;
+    return pl.nt == 1 ? launch_nt<1>(pl, p, map_k, map_v, bh, stream) : launch_nt<2>(pl, p, map_k, map_v, bh, stream);
+}
+
+}  // namespace ec

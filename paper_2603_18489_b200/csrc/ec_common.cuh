@@ -69,6 +69,10 @@ struct AttendArgs {
 size_t attend_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_f32(const AttendArgs& a, cudaStream_t stream);
 cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);      // mma.sync path (any head_dim)
+// fused skip-step path (bf16, head_dim 128, n_active * H_q/H_kv <= 256): refresh + attention + merge in one launch
+bool attend_skip_supported(const ec_attn_desc& d, int n_active);
+cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
+                               cudaStream_t stream);
 size_t attend_tc_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_bf16_tc(const AttendArgs& a, cudaStream_t stream);   // tcgen05 path (head_dim 128)
 
