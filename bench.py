@@ -457,24 +457,17 @@ def run_cuda(args) -> None:
 
 
 def _run_only(args, torch, w, n_layers: int, dev) -> None:
-    """Profiling aid: plain (non-graph) launches of one part of the step over the same
-    device workload, a few iterations, one short JSON line.  Not a benchmark figure."""
+    """Profiling aid: one part of the step over the same device workload (one CUDA graph
+    per step, like the full run), a few iterations, one short JSON line."""
     wl = DeviceWorkload(w, n_layers, dev, seed=1234, need_recompute=args.only == "recompute")
     body = {"skip": lambda: [wl.attend_skip(l) for l in range(n_layers)],
             "recompute": lambda: [wl.attend_recompute(l) for l in range(n_layers)],
             "gate": lambda: [wl.gate(i) for i in range(wl.n_lbuf)]}[args.only]
     calls = wl.n_lbuf if args.only == "gate" else n_layers
-    for _ in range(max(args.warmup, 1)):
-        body()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        body()
-    e1.record()
-    torch.cuda.synchronize()
-    print(json.dumps({"only": args.only, "workload": w.name, "calls_per_iteration": calls,
-                      "us_per_call_eager": e0.elapsed_time(e1) * 1e3 / (args.steps * calls)}))
+    stream = torch.cuda.Stream(device=dev)
+    ms = _graph_time(torch, body, max(args.steps, 1), max(args.warmup, 1), stream)
+    print(json.dumps({"only": args.only, "workload": w.name, "calls_per_step": calls,
+                      "us_per_call": ms * 1e3 / calls}))
 
 
 def main() -> None:
@@ -486,7 +479,7 @@ def main() -> None:
     ap.add_argument("--layers", type=int, default=0, help="distinct K/V caches per step (0: enough to exceed 3x L2)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--only", default="", choices=["", "skip", "recompute", "gate"],
-                    help="profiling aid: run only this part of the step with plain launches")
+                    help="profiling aid: run only this part of the step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
