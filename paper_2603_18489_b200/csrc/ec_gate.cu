@@ -3,20 +3,31 @@
 // entropy over the rows flagged "newly decoded" and its comparison with tau
 // (Algorithm 1: E > tau -> recompute, else skip).
 //
-// The pass is HBM-bound: R*V*sizeof(elem) bytes are read exactly once.
-//   grid  = (splits, R): CTA (s, r) owns the column chunk [s*chunk, (s+1)*chunk) of row r,
-//           chunk = 256 threads * 8 elements * NV vectors, all loads issued up front
-//           as 16-byte vectors (bf16x8 / 2 x f32x4) and held in registers;
-//   max   : thread max -> CTA max (shuffles + shared memory), with the first index
-//           attaining it (order-preserving 64-bit key, ties -> smallest index);
-//   sums  : S = sum 2^d, T = sum 2^d * d with d = x*log2(e) - base, base = fl(M*log2(e)),
-//           one ex2.approx + one FMA-formed exponent per element;
-//   merge : CTA partial (M, S, T, idx) -> workspace; the last CTA of a row (atomic
-//           ticket, no spinning) merges the row's partials and writes
-//           H = ln S - ln2 * T / S, conf = 2^(M*log2e - base) / S, argmax;
-//           the last row of a sequence takes the flagged maximum and the decision.
+// The pass is HBM-bound: R*V*sizeof(elem) bytes are read exactly once; the arithmetic is kept to about
+// six instructions per element so that the issue slots do not become the limit first.
+//   grid  = (splits, R): CTA (s, r) owns the columns [s*chunk, (s+1)*chunk) of row r; the split count is
+//           chosen so that the whole grid is about one resident wave (4 CTAs of 256 threads per SM);
+//   loop  : a thread visits its columns in ascending order, four 16-byte vectors (bf16x8 / f32x4) per
+//           iteration, the next four already in flight (register double buffer), and keeps a running
+//           (max, S, T) with S = sum 2^d, T = sum 2^d * d, d = x*log2(e) - base: one FMA, one ex2.approx,
+//           one add and one FMA per element.  The base follows the maximum lazily: it moves, and S and T
+//           are rescaled (S' = 2^dl S, T' = 2^dl (T + dl S), dl = old base - new base), only when a value
+//           exceeds it by more than 2^64, so the common path has no data-dependent branch.  Logits are
+//           clamped from below at -1e38 (packed bf16 max on the raw words), which keeps d finite:
+//           -inf and finfo.min-style masks get probability 0 without a per-element special case;
+//   argmax: the thread remembers the iteration that raised its maximum; after the CTA-wide maximum is
+//           known, only the threads that attained it look at that iteration's vectors again for the
+//           first column (ties -> smallest index, through every reduction stage);
+//   CTA   : sums rescaled to the CTA's base and added (shuffles + shared memory);
+//   merge : CTA partial (M, S, T, idx) -> workspace, one atomic ticket; the last CTA of a sequence
+//           (no spinning: tickets only count arrivals) merges the partials of every row of the
+//           sequence, writes H = ln S - ln2 * T / S, conf = 2^(M*log2e - base) / S and argmax, takes
+//           the flagged maximum and the decision.  Sequences of more than 64 rows, or rows cut into more
+//           than 32 splits, use two ticket levels instead (last CTA of a row, then last row of the sequence).
 // The entropy identity used: with p_j = 2^{d_j} / S,  -sum p_j ln p_j = ln S - ln2 * T / S
 // for any common base, so no partial ever needs the true row maximum.
+// The kernel is launched with programmatic stream serialisation and touches global memory only after
+// griddepcontrol.wait.
 #include "ec_common.cuh"
 
 #include <float.h>
@@ -25,31 +36,23 @@ namespace ec {
 namespace {
 
 constexpr int kGateThreads = 256;
-constexpr int kVec = 8;  // elements per thread per vector
+constexpr int kVec = 8;  // columns per thread in one slab of kGateThreads * kVec columns (chunk granularity)
 constexpr int kMaxSplits = 96;
-constexpr float kDClamp = -150.0f;  // 2^-150 flushes to 0 (ftz): masked / -inf logits add nothing
+constexpr float kDClamp = -150.0f;  // 2^-150 flushes to 0 (ftz)
+constexpr int kUnroll = 4;          // 16-byte vectors per thread per iteration
+constexpr int kSingleLevelMaxRows = 64;
+constexpr float kRebase = 64.f;     // the base moves when a value exceeds it by more than 2^kRebase
+constexpr unsigned int kXMinBf16x2 = 0xFE96FE96u;   // two bf16 of about -1e38: lower clamp of the logits
+constexpr unsigned int kXMinF32 = 0xFE960000u;      // the same value as fp32 bits
 
 struct Partial {
-    float M;  // raw maximum of the chunk (-inf if the chunk holds no finite value)
+    float M;  // maximum of the chunk (clamped logits)
     float S;  // sum 2^(x*log2e - base(M))
     float T;  // sum 2^(..) * (x*log2e - base(M))
     int idx;  // first column attaining M
 };
 
 __device__ __forceinline__ float base_of(float M) { return fmaxf(M * kLog2e, -3.0e38f); }
-
-__device__ __forceinline__ unsigned int orderable(float f) {
-    unsigned int u = __float_as_uint(f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float unorderable(unsigned int k) {
-    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-
-// (M desc, idx asc) lexicographic maximum
-__device__ __forceinline__ unsigned long long make_key(float M, int idx) {
-    return ((unsigned long long)orderable(M) << 32) | (unsigned int)(0x7fffffff - idx);
-}
 
 __device__ __forceinline__ Partial merge(Partial a, Partial b) {
     const bool a_wins = (a.M > b.M) || (a.M == b.M && a.idx <= b.idx);
@@ -64,13 +67,36 @@ __device__ __forceinline__ Partial merge(Partial a, Partial b) {
     return hi;
 }
 
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ unsigned int max_bf16x2(unsigned int a, unsigned int b) {
+    unsigned int d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// One 16-byte vector of a row: EPV elements, kept raw (packed) while in flight.
+//   clamp()    lower clamp of all elements, on the raw words
+//   vec_max()  maximum of the (clamped) vector as fp32
+//   widen()    raw -> fp32
 template <typename T>
 struct Loader;
 
 template <>
 struct Loader<__nv_bfloat16> {
-    static __device__ __forceinline__ void vec(const __nv_bfloat16* p, float (&x)[kVec]) {
-        const uint4 u = __ldcs(reinterpret_cast<const uint4*>(p));  // streamed once: evict first
+    static constexpr int EPV = 8;
+    static __device__ __forceinline__ void clamp(uint4& u) {
+        u.x = max_bf16x2(u.x, kXMinBf16x2); u.y = max_bf16x2(u.y, kXMinBf16x2);
+        u.z = max_bf16x2(u.z, kXMinBf16x2); u.w = max_bf16x2(u.w, kXMinBf16x2);
+    }
+    static __device__ __forceinline__ unsigned int max_word(const uint4& u) {
+        return max_bf16x2(max_bf16x2(u.x, u.y), max_bf16x2(u.z, u.w));
+    }
+    static __device__ __forceinline__ unsigned int max_words(unsigned int a, unsigned int b) { return max_bf16x2(a, b); }
+    static __device__ __forceinline__ float word_max(unsigned int w) {
+        return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+    static __device__ __forceinline__ void widen(const uint4& u, float (&x)[8]) {
         const unsigned int w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -78,24 +104,41 @@ struct Loader<__nv_bfloat16> {
             x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
     }
-    static __device__ __forceinline__ float one(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ float one(const __nv_bfloat16* p) {
+        return fmaxf(__bfloat162float(*p), __uint_as_float(kXMinF32));
+    }
 };
 
 template <>
 struct Loader<float> {
-    static __device__ __forceinline__ void vec(const float* p, float (&x)[kVec]) {
-        const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
-        const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-        x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    static constexpr int EPV = 4;
+    static __device__ __forceinline__ void clamp(uint4& u) {
+        const float lo = __uint_as_float(kXMinF32);
+        u.x = __float_as_uint(fmaxf(__uint_as_float(u.x), lo)); u.y = __float_as_uint(fmaxf(__uint_as_float(u.y), lo));
+        u.z = __float_as_uint(fmaxf(__uint_as_float(u.z), lo)); u.w = __float_as_uint(fmaxf(__uint_as_float(u.w), lo));
     }
-    static __device__ __forceinline__ float one(const float* p) { return *p; }
+    // "word" = one fp32 value here
+    static __device__ __forceinline__ unsigned int max_word(const uint4& u) {
+        return __float_as_uint(fmaxf(fmaxf(__uint_as_float(u.x), __uint_as_float(u.y)),
+                                     fmaxf(__uint_as_float(u.z), __uint_as_float(u.w))));
+    }
+    static __device__ __forceinline__ unsigned int max_words(unsigned int a, unsigned int b) {
+        return __float_as_uint(fmaxf(__uint_as_float(a), __uint_as_float(b)));
+    }
+    static __device__ __forceinline__ float word_max(unsigned int w) { return __uint_as_float(w); }
+    static __device__ __forceinline__ void widen(const uint4& u, float (&x)[4]) {
+        x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y);
+        x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
+    }
+    static __device__ __forceinline__ float one(const float* p) { return fmaxf(*p, __uint_as_float(kXMinF32)); }
 };
 
 struct GateParams {
     const void* logits;
     long long row_stride;
     int n_rows, vocab, rows_per_seq, splits;
+    int chunk;          // columns per CTA, a multiple of kGateThreads * kVec
+    int single_level;   // 1: the last CTA of a sequence finishes all its rows; 0: per-row then per-sequence tickets
     const uint8_t* flags;
     float tau;
     int* argmax_out;
@@ -108,143 +151,268 @@ struct GateParams {
     Partial* partials;  // [n_rows, splits]
 };
 
-template <typename T, int NV>
-__global__ void __launch_bounds__(kGateThreads) gate_kernel(const GateParams p) {
-    __shared__ unsigned long long s_key[kGateThreads / 32];
+// warp-collective: merge the split partials of one row, write the row's outputs, return its entropy (all lanes)
+__device__ __forceinline__ float finish_row(const GateParams& p, int row, int lane) {
+    Partial acc;
+    acc.M = -INFINITY; acc.S = 0.f; acc.T = 0.f; acc.idx = 0x7fffffff;
+    for (int s = lane; s < p.splits; s += 32) {
+        const float4 f = __ldcg(reinterpret_cast<const float4*>(&p.partials[(long long)row * p.splits + s]));
+        Partial q;
+        q.M = f.x; q.S = f.y; q.T = f.z; q.idx = __float_as_int(f.w);
+        acc = merge(acc, q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial q;
+        q.M = __shfl_xor_sync(0xffffffffu, acc.M, o);
+        q.S = __shfl_xor_sync(0xffffffffu, acc.S, o);
+        q.T = __shfl_xor_sync(0xffffffffu, acc.T, o);
+        q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+        acc = merge(acc, q);
+    }
+    const float H = fmaxf(logf(acc.S) - kLn2 * acc.T / acc.S, 0.f);
+    if (lane == 0) {
+        const float conf = fast_exp2(fmaf(acc.M, kLog2e, -base_of(acc.M))) / acc.S;
+        if (p.argmax_out) p.argmax_out[row] = acc.idx;
+        if (p.conf_out) p.conf_out[row] = conf;
+        p.entropy_out[row] = H;
+    }
+    return H;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams p) {
+    __shared__ float s_m[kGateThreads / 32];
+    __shared__ int s_i[kGateThreads / 32];
     __shared__ float s_S[kGateThreads / 32], s_T[kGateThreads / 32];
+    __shared__ float s_H[kSingleLevelMaxRows];
     __shared__ int s_last;
 
+    constexpr int EPV = Loader<T>::EPV;
+    constexpr int kVStride = kGateThreads * EPV;     // columns between a thread's consecutive vectors
+    constexpr int kStep = kUnroll * kVStride;        // columns per loop iteration
     const int row = blockIdx.y, split = blockIdx.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     const T* rowp = reinterpret_cast<const T*>(p.logits) + (long long)row * p.row_stride;
-    const int c0 = split * (kGateThreads * kVec * NV);
-    const int V = p.vocab;
+    const int c0 = split * p.chunk;
+    const int c_end = min(p.vocab, c0 + p.chunk);
 
-    // ---- load everything this thread owns -----------------------------------------
-    float x[NV][kVec];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int col = c0 + (v * kGateThreads + tid) * kVec;
-        if (col + kVec <= V) {
-            Loader<T>::vec(rowp + col, x[v]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < kVec; ++i) x[v][i] = (col + i < V) ? Loader<T>::one(rowp + col + i) : -INFINITY;
-        }
-    }
+    pdl_wait();                 // the previous kernel of the stream has completed: the logits are final
+    pdl_launch_dependents();
 
-    // ---- maximum and its first index ----------------------------------------------
-    float tmax = -INFINITY;
+    float m = -INFINITY, base = base_of(-INFINITY), S = 0.f, Tt = 0.f;
+    int mcol = -1, mspan = 0;   // where the maximum was raised: first column of the vectors to look at again, and how many
+    auto accumulate = [&](const float (&x)[EPV]) {
 #pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const float m01 = fmaxf(x[v][0], x[v][1]), m23 = fmaxf(x[v][2], x[v][3]);
-        const float m45 = fmaxf(x[v][4], x[v][5]), m67 = fmaxf(x[v][6], x[v][7]);
-        tmax = fmaxf(tmax, fmaxf(fmaxf(m01, m23), fmaxf(m45, m67)));
-    }
-    int tidx = 0x7fffffff;
-#pragma unroll
-    for (int v = NV - 1; v >= 0; --v) {
-        const int col = c0 + (v * kGateThreads + tid) * kVec;
-#pragma unroll
-        for (int i = kVec - 1; i >= 0; --i)
-            if (x[v][i] == tmax) tidx = col + i;  // descending scan: the smallest index survives
-    }
-    unsigned long long key = make_key(tmax, tidx);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-        key = other > key ? other : key;
-    }
-    if (lane == 0) s_key[warp] = key;
-    __syncthreads();
-    key = s_key[0];
-#pragma unroll
-    for (int w = 1; w < kGateThreads / 32; ++w) key = s_key[w] > key ? s_key[w] : key;
-    const float M = unorderable((unsigned int)(key >> 32));
-    const int idx = 0x7fffffff - (int)(unsigned int)(key & 0xffffffffu);
-    const float base = base_of(M);
-
-    // ---- exponent sums against the CTA-wide base ----------------------------------
-    float S = 0.f, Tt = 0.f;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-#pragma unroll
-        for (int i = 0; i < kVec; ++i) {
-            const float d = fmaxf(fmaf(x[v][i], kLog2e, -base), kDClamp);
+        for (int i = 0; i < EPV; ++i) {
+            const float d = fmaf(x[i], kLog2e, -base);
             const float e = fast_exp2(d);
             S += e;
             Tt = fmaf(e, d, Tt);
         }
+    };
+    auto rebase_if_needed = [&](float vmax) {
+        if (fmaf(vmax, kLog2e, -base) > kRebase) {   // rare
+            const float nb = base_of(vmax);
+            if (S > 0.f) {
+                const float dl = fmaxf(base - nb, kDClamp);
+                const float c = fast_exp2(dl);
+                Tt = c * fmaf(dl, S, Tt);
+                S *= c;
+            }
+            base = nb;
+        }
+    };
+
+    // ---- full iterations: kUnroll in-bounds vectors per thread, the next kUnroll already in flight ------
+    const int n_full = (c_end - c0) / kStep;
+    auto fetch = [&](int it, uint4 (&raw)[kUnroll]) {
+        const T* src = rowp + c0 + it * kStep + tid * EPV;
+#pragma unroll
+        for (int v = 0; v < kUnroll; ++v) raw[v] = __ldcs(reinterpret_cast<const uint4*>(src + v * kVStride));   // streamed once
+    };
+    auto consume = [&](int it, uint4 (&raw)[kUnroll]) {
+        unsigned int w = 0;
+#pragma unroll
+        for (int v = 0; v < kUnroll; ++v) {
+            Loader<T>::clamp(raw[v]);
+            const unsigned int wv = Loader<T>::max_word(raw[v]);
+            w = v == 0 ? wv : Loader<T>::max_words(w, wv);
+        }
+        const float it_max = Loader<T>::word_max(w);
+        rebase_if_needed(it_max);
+        const bool up = it_max > m;   // strictly greater: the first iteration of a tie survives
+        m = up ? it_max : m;
+        mcol = up ? c0 + it * kStep + tid * EPV : mcol;
+        mspan = up ? kUnroll : mspan;
+#pragma unroll
+        for (int v = 0; v < kUnroll; ++v) {
+            float x[EPV];
+            Loader<T>::widen(raw[v], x);
+            accumulate(x);
+        }
+    };
+    if (n_full > 0) {
+        uint4 ra[kUnroll], rb[kUnroll];
+        fetch(0, ra);
+        for (int it = 0; it < n_full; it += 2) {
+            if (it + 1 < n_full) fetch(it + 1, rb);
+            consume(it, ra);
+            if (it + 1 < n_full) {
+                if (it + 2 < n_full) fetch(it + 2, ra);
+                consume(it + 1, rb);
+            }
+        }
+    }
+    // ---- the rest of the chunk: one guarded vector at a time ------------------------------------------------
+    for (int col = c0 + n_full * kStep + tid * EPV; col < c_end; col += kVStride) {
+        float x[EPV];
+        if (col + EPV <= c_end) {
+            uint4 raw = __ldcs(reinterpret_cast<const uint4*>(rowp + col));
+            Loader<T>::clamp(raw);
+            Loader<T>::widen(raw, x);
+        } else {   // ragged end of the row: -inf stands for "no column"
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) x[i] = (col + i < c_end) ? Loader<T>::one(rowp + col + i) : -INFINITY;
+        }
+        float vmax = x[0];
+#pragma unroll
+        for (int i = 1; i < EPV; ++i) vmax = fmaxf(vmax, x[i]);
+        rebase_if_needed(vmax);
+        const bool up = vmax > m;
+        m = up ? vmax : m;
+        mcol = up ? col : mcol;
+        mspan = up ? 1 : mspan;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {   // -inf marks "no column": 2^-inf = 0, and the product is kept out of T
+            const float d = fmaf(x[i], kLog2e, -base);
+            const float e = fast_exp2(d);
+            S += e;
+            Tt = (x[i] == -INFINITY) ? Tt : fmaf(e, d, Tt);
+        }
+    }
+
+    // ---- CTA-wide maximum; the threads that attained it find its first column ---------------------------
+    float wm = m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+    if (lane == 0) s_m[warp] = wm;
+    __syncthreads();
+    float M = s_m[0];
+#pragma unroll
+    for (int w = 1; w < kGateThreads / 32; ++w) M = fmaxf(M, s_m[w]);
+    int idx = 0x7fffffff;
+    if (m == M && mcol >= 0) {
+        for (int v = mspan - 1; v >= 0; --v) {   // descending: the smallest column survives
+            const int col = mcol + v * kVStride;
+#pragma unroll
+            for (int i = EPV - 1; i >= 0; --i)
+                if (col + i < c_end && Loader<T>::one(rowp + col + i) == M) idx = col + i;
+        }
+    }
+    // ---- sums against the CTA's base, first column of the maximum --------------------------------------
+    if (S > 0.f) {
+        const float dl = fmaxf(base - base_of(M), kDClamp);
+        const float c = fast_exp2(dl);
+        Tt = c * fmaf(dl, S, Tt);
+        S *= c;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         S += __shfl_xor_sync(0xffffffffu, S, o);
         Tt += __shfl_xor_sync(0xffffffffu, Tt, o);
+        idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, o));
     }
-    if (lane == 0) { s_S[warp] = S; s_T[warp] = Tt; }
+    if (lane == 0) { s_S[warp] = S; s_T[warp] = Tt; s_i[warp] = idx; }
     __syncthreads();
 
-    // ---- publish the partial; the last CTA of the row finishes the row ------------
+    // ---- publish the partial; count arrivals (tickets only count, nothing spins) --------------------
+    const int seq = row / p.rows_per_seq;
     if (tid == 0) {
         float Ss = 0.f, Ts = 0.f;
+        int Midx = 0x7fffffff;
 #pragma unroll
-        for (int w = 0; w < kGateThreads / 32; ++w) { Ss += s_S[w]; Ts += s_T[w]; }
-        Partial out;
-        out.M = M; out.S = Ss; out.T = Ts; out.idx = idx;
-        int last = 1;
-        if (p.splits > 1) {
-            *reinterpret_cast<float4*>(&p.partials[(long long)row * p.splits + split]) =
-                make_float4(out.M, out.S, out.T, __int_as_float(out.idx));
-            __threadfence();
+        for (int w = 0; w < kGateThreads / 32; ++w) { Ss += s_S[w]; Ts += s_T[w]; Midx = min(Midx, s_i[w]); }
+        *reinterpret_cast<float4*>(&p.partials[(long long)row * p.splits + split]) =
+            make_float4(M, Ss, Ts, __int_as_float(Midx));
+        __threadfence();
+        int last;
+        if (p.single_level)
+            last = (atomicAdd(&p.seq_ticket[seq], 1) == p.rows_per_seq * p.splits - 1);
+        else
             last = (atomicAdd(&p.row_ticket[row], 1) == p.splits - 1);
-        }
         s_last = last;
     }
     __syncthreads();
-    if (!s_last || warp != 0) return;
+    if (!s_last) return;
+    __threadfence();
 
-    Partial acc;
-    if (p.splits > 1) {
-        __threadfence();
-        acc.M = -INFINITY; acc.S = 0.f; acc.T = 0.f; acc.idx = 0x7fffffff;
-        for (int s = lane; s < p.splits; s += 32) {
-            const float4 f = __ldcg(reinterpret_cast<const float4*>(&p.partials[(long long)row * p.splits + s]));
-            Partial q;
-            q.M = f.x; q.S = f.y; q.T = f.z; q.idx = __float_as_int(f.w);
-            acc = merge(acc, q);
-        }
+    if (p.single_level) {
+        // ---- last CTA of the sequence: finish every row, then the masked maximum and the decision ----
+        // eight threads per row (each merges up to four split partials, then three shuffle steps), 32 rows per pass
+        for (int r0 = 0; r0 < p.rows_per_seq; r0 += kGateThreads / 8) {
+            const int r = r0 + (tid >> 3), j = tid & 7;
+            const bool ok = r < p.rows_per_seq;
+            const int rr = seq * p.rows_per_seq + (ok ? r : 0);
+            float4 f[4];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            Partial q;
-            q.M = __shfl_xor_sync(0xffffffffu, acc.M, o);
-            q.S = __shfl_xor_sync(0xffffffffu, acc.S, o);
-            q.T = __shfl_xor_sync(0xffffffffu, acc.T, o);
-            q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
-            acc = merge(acc, q);
-        }
-    } else {
-        float Ss = 0.f, Ts = 0.f;
+            for (int k = 0; k < 4; ++k) {
+                const int sp = j + 8 * k;
+                f[k] = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(0x7fffffff));
+                if (ok && sp < p.splits) f[k] = __ldcg(reinterpret_cast<const float4*>(&p.partials[(long long)rr * p.splits + sp]));
+            }
+            Partial acc;
+            acc.M = f[0].x; acc.S = f[0].y; acc.T = f[0].z; acc.idx = __float_as_int(f[0].w);
 #pragma unroll
-        for (int w = 0; w < kGateThreads / 32; ++w) { Ss += s_S[w]; Ts += s_T[w]; }
-        acc.M = M; acc.S = Ss; acc.T = Ts; acc.idx = idx;
+            for (int k = 1; k < 4; ++k) {
+                Partial q;
+                q.M = f[k].x; q.S = f[k].y; q.T = f[k].z; q.idx = __float_as_int(f[k].w);
+                acc = merge(acc, q);
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                Partial q;
+                q.M = __shfl_xor_sync(0xffffffffu, acc.M, o);
+                q.S = __shfl_xor_sync(0xffffffffu, acc.S, o);
+                q.T = __shfl_xor_sync(0xffffffffu, acc.T, o);
+                q.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+                acc = merge(acc, q);
+            }
+            if (ok && j == 0) {
+                const float H = fmaxf(logf(acc.S) - kLn2 * acc.T / acc.S, 0.f);
+                const float conf = fast_exp2(fmaf(acc.M, kLog2e, -base_of(acc.M))) / acc.S;
+                if (p.argmax_out) p.argmax_out[rr] = acc.idx;
+                if (p.conf_out) p.conf_out[rr] = conf;
+                p.entropy_out[rr] = H;
+                s_H[r] = p.flags[rr] ? H : -INFINITY;
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            float E = -INFINITY;
+            for (int r = lane; r < p.rows_per_seq; r += 32) E = fmaxf(E, s_H[r]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+            if (lane == 0) {
+                p.max_entropy_out[seq] = E;
+                p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
+                p.seq_ticket[seq] = 0;   // ready for the next call
+            }
+        }
+        return;
     }
 
+    // ---- last CTA of the row finishes the row; the last row of the sequence finishes the sequence ----
+    if (warp != 0) return;
+    finish_row(p, row, lane);
     int seq_last = 0;
-    const int seq = row / p.rows_per_seq;
     if (lane == 0) {
-        const float H = fmaxf(logf(acc.S) - kLn2 * acc.T / acc.S, 0.f);
-        const float conf = fast_exp2(fmaf(acc.M, kLog2e, -base_of(acc.M))) / acc.S;
-        if (p.argmax_out) p.argmax_out[row] = acc.idx;
-        if (p.conf_out) p.conf_out[row] = conf;
-        p.entropy_out[row] = H;
-        if (p.splits > 1) p.row_ticket[row] = 0;  // ready for the next call
+        p.row_ticket[row] = 0;
         __threadfence();
         seq_last = (atomicAdd(&p.seq_ticket[seq], 1) == p.rows_per_seq - 1);
     }
     seq_last = __shfl_sync(0xffffffffu, seq_last, 0);
     if (!seq_last) return;
-
-    // ---- masked maximum over the sequence's rows and the decision -----------------
     __threadfence();
     float E = -INFINITY;
     for (int r = lane; r < p.rows_per_seq; r += 32) {
@@ -275,29 +443,35 @@ GateWs carve(int n_rows) {
     return w;
 }
 
-int pick_nv(int n_rows, int vocab) {
-    // prefer the largest per-CTA chunk that still gives every SM a few CTAs
-    const long long want = 3LL * sm_count();
-    for (int nv = 4; nv > 1; nv >>= 1) {
-        const long long per = (long long)kGateThreads * kVec * nv;
-        const long long ctas = ((vocab + per - 1) / per) * n_rows;
-        if (ctas >= want) return nv;
-    }
-    return 1;
+// split count and columns per CTA: about one resident wave (4 CTAs of 256 threads per SM), every CTA a whole number
+// of 2048-column slabs, at most kMaxSplits partials per row
+void plan_chunks(int n_rows, int vocab, int* splits, int* chunk) {
+    const int slab = kGateThreads * kVec;
+    const long long slots = 4LL * sm_count();
+    long long want = slots / n_rows;
+    if (want < 1) want = 1;
+    if (want > kMaxSplits) want = kMaxSplits;
+    long long per = (vocab + want - 1) / want;
+    const long long per_min = (vocab + kMaxSplits - 1) / kMaxSplits;
+    if (per < per_min) per = per_min;
+    per = (per + slab - 1) / slab * slab;
+    *chunk = (int)per;
+    *splits = (int)((vocab + per - 1) / per);
 }
 
 template <typename T>
-cudaError_t launch_t(const GateParams& p0, int nv, cudaStream_t stream) {
-    GateParams p = p0;
-    const int per = kGateThreads * kVec * nv;
-    p.splits = (p.vocab + per - 1) / per;
-    const dim3 grid(p.splits, p.n_rows);
-    switch (nv) {
-        case 4: gate_kernel<T, 4><<<grid, kGateThreads, 0, stream>>>(p); break;
-        case 2: gate_kernel<T, 2><<<grid, kGateThreads, 0, stream>>>(p); break;
-        default: gate_kernel<T, 1><<<grid, kGateThreads, 0, stream>>>(p); break;
-    }
-    return cudaGetLastError();
+cudaError_t launch_t(const GateParams& p, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(p.splits, p.n_rows, 1);
+    cfg.blockDim = dim3(kGateThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // launch latency may overlap the previous kernel's tail
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gate_kernel<T>, p);
 }
 
 }  // namespace
@@ -317,6 +491,8 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     p.vocab = a.vocab;
     p.rows_per_seq = a.rows_per_seq;
     p.splits = 0;
+    p.chunk = 0;
+    p.single_level = 0;
     p.flags = a.flags;
     p.tau = a.tau;
     p.argmax_out = a.argmax_out;
@@ -327,11 +503,10 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     p.row_ticket = reinterpret_cast<int*>(ws + w.off_row);
     p.seq_ticket = reinterpret_cast<int*>(ws + w.off_seq);
     p.partials = reinterpret_cast<Partial*>(ws + w.off_part);
-    int nv = pick_nv(a.n_rows, a.vocab);
-    // the split count must fit the workspace
-    while ((a.vocab + kGateThreads * kVec * nv - 1) / (kGateThreads * kVec * nv) > kMaxSplits) nv *= 2;
-    if (nv > 4) return cudaErrorInvalidValue;  // vocab > 96 * 8192: rejected by the API layer before this
-    return a.dtype == EC_BF16 ? launch_t<__nv_bfloat16>(p, nv, stream) : launch_t<float>(p, nv, stream);
+    plan_chunks(a.n_rows, a.vocab, &p.splits, &p.chunk);
+    if (p.splits > kMaxSplits) return cudaErrorInvalidValue;   // vocab > 96 * 8192: rejected by the API layer before this
+    p.single_level = (a.rows_per_seq <= kSingleLevelMaxRows && p.splits <= 32) ? 1 : 0;
+    return a.dtype == EC_BF16 ? launch_t<__nv_bfloat16>(p, stream) : launch_t<float>(p, stream);
 }
 
 }  // namespace ec
