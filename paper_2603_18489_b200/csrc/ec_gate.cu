@@ -224,71 +224,84 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
         }
     };
 
-    // ---- full iterations: kUnroll in-bounds vectors per thread, the next kUnroll already in flight ------
+    // ---- kUnroll vectors per thread per iteration, the next kUnroll already in flight ------------------------
+    // Only the chunk's last iteration can hold vectors that are ragged or past the end; it takes the guarded path.
     const int n_full = (c_end - c0) / kStep;
+    const int n_iter = (c_end - c0 + kStep - 1) / kStep;
     auto fetch = [&](int it, uint4 (&raw)[kUnroll]) {
-        const T* src = rowp + c0 + it * kStep + tid * EPV;
+        const int col0 = c0 + it * kStep + tid * EPV;
+        if (it < n_full) {
 #pragma unroll
-        for (int v = 0; v < kUnroll; ++v) raw[v] = __ldcs(reinterpret_cast<const uint4*>(src + v * kVStride));   // streamed once
+            for (int v = 0; v < kUnroll; ++v) raw[v] = __ldcs(reinterpret_cast<const uint4*>(rowp + col0 + v * kVStride));   // streamed once
+        } else {
+#pragma unroll
+            for (int v = 0; v < kUnroll; ++v)
+                if (col0 + v * kVStride + EPV <= c_end) raw[v] = __ldcs(reinterpret_cast<const uint4*>(rowp + col0 + v * kVStride));
+        }
     };
     auto consume = [&](int it, uint4 (&raw)[kUnroll]) {
-        unsigned int w = 0;
+        const int col0 = c0 + it * kStep + tid * EPV;
+        if (it < n_full) {
+            unsigned int w = 0;
 #pragma unroll
-        for (int v = 0; v < kUnroll; ++v) {
-            Loader<T>::clamp(raw[v]);
-            const unsigned int wv = Loader<T>::max_word(raw[v]);
-            w = v == 0 ? wv : Loader<T>::max_words(w, wv);
-        }
-        const float it_max = Loader<T>::word_max(w);
-        rebase_if_needed(it_max);
-        const bool up = it_max > m;   // strictly greater: the first iteration of a tie survives
-        m = up ? it_max : m;
-        mcol = up ? c0 + it * kStep + tid * EPV : mcol;
-        mspan = up ? kUnroll : mspan;
+            for (int v = 0; v < kUnroll; ++v) {
+                Loader<T>::clamp(raw[v]);
+                const unsigned int wv = Loader<T>::max_word(raw[v]);
+                w = v == 0 ? wv : Loader<T>::max_words(w, wv);
+            }
+            const float it_max = Loader<T>::word_max(w);
+            rebase_if_needed(it_max);
+            const bool up = it_max > m;   // strictly greater: the first iteration of a tie survives
+            m = up ? it_max : m;
+            mcol = up ? col0 : mcol;
+            mspan = up ? kUnroll : mspan;
 #pragma unroll
-        for (int v = 0; v < kUnroll; ++v) {
-            float x[EPV];
-            Loader<T>::widen(raw[v], x);
-            accumulate(x);
-        }
-    };
-    if (n_full > 0) {
-        uint4 ra[kUnroll], rb[kUnroll];
-        fetch(0, ra);
-        for (int it = 0; it < n_full; it += 2) {
-            if (it + 1 < n_full) fetch(it + 1, rb);
-            consume(it, ra);
-            if (it + 1 < n_full) {
-                if (it + 2 < n_full) fetch(it + 2, ra);
-                consume(it + 1, rb);
+            for (int v = 0; v < kUnroll; ++v) {
+                float x[EPV];
+                Loader<T>::widen(raw[v], x);
+                accumulate(x);
+            }
+        } else {
+#pragma unroll
+            for (int v = 0; v < kUnroll; ++v) {
+                const int col = col0 + v * kVStride;
+                if (col >= c_end) continue;
+                float x[EPV];
+                if (col + EPV <= c_end) {
+                    Loader<T>::clamp(raw[v]);
+                    Loader<T>::widen(raw[v], x);
+                } else {   // ragged end of the row: -inf stands for "no column"
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) x[i] = (col + i < c_end) ? Loader<T>::one(rowp + col + i) : -INFINITY;
+                }
+                float vmax = x[0];
+#pragma unroll
+                for (int i = 1; i < EPV; ++i) vmax = fmaxf(vmax, x[i]);
+                rebase_if_needed(vmax);
+                const bool up = vmax > m;
+                m = up ? vmax : m;
+                mcol = up ? col : mcol;
+                mspan = up ? 1 : mspan;
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) {   // 2^-inf = 0, and that product is kept out of T
+                    const float d = fmaf(x[i], kLog2e, -base);
+                    const float e = fast_exp2(d);
+                    S += e;
+                    Tt = (x[i] == -INFINITY) ? Tt : fmaf(e, d, Tt);
+                }
             }
         }
-    }
-    // ---- the rest of the chunk: one guarded vector at a time ------------------------------------------------
-    for (int col = c0 + n_full * kStep + tid * EPV; col < c_end; col += kVStride) {
-        float x[EPV];
-        if (col + EPV <= c_end) {
-            uint4 raw = __ldcs(reinterpret_cast<const uint4*>(rowp + col));
-            Loader<T>::clamp(raw);
-            Loader<T>::widen(raw, x);
-        } else {   // ragged end of the row: -inf stands for "no column"
-#pragma unroll
-            for (int i = 0; i < EPV; ++i) x[i] = (col + i < c_end) ? Loader<T>::one(rowp + col + i) : -INFINITY;
-        }
-        float vmax = x[0];
-#pragma unroll
-        for (int i = 1; i < EPV; ++i) vmax = fmaxf(vmax, x[i]);
-        rebase_if_needed(vmax);
-        const bool up = vmax > m;
-        m = up ? vmax : m;
-        mcol = up ? col : mcol;
-        mspan = up ? 1 : mspan;
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) {   // -inf marks "no column": 2^-inf = 0, and the product is kept out of T
-            const float d = fmaf(x[i], kLog2e, -base);
-            const float e = fast_exp2(d);
-            S += e;
-            Tt = (x[i] == -INFINITY) ? Tt : fmaf(e, d, Tt);
+    };
+    {
+        uint4 ra[kUnroll], rb[kUnroll];
+        fetch(0, ra);
+        for (int it = 0; it < n_iter; it += 2) {
+            if (it + 1 < n_iter) fetch(it + 1, rb);
+            consume(it, ra);
+            if (it + 1 < n_iter) {
+                if (it + 2 < n_iter) fetch(it + 2, ra);
+                consume(it + 1, rb);
+            }
         }
     }
 
@@ -454,7 +467,8 @@ void plan_chunks(int n_rows, int vocab, int* splits, int* chunk) {
     long long per = (vocab + want - 1) / want;
     const long long per_min = (vocab + kMaxSplits - 1) / kMaxSplits;
     if (per < per_min) per = per_min;
-    per = (per + slab - 1) / slab * slab;
+    const long long step = (long long)kUnroll * slab;   // one loop iteration of the bf16 kernel
+    per = per >= 2 * step ? (per + step - 1) / step * step : (per + slab - 1) / slab * slab;
     *chunk = (int)per;
     *splits = (int)((vocab + per - 1) / per);
 }
