@@ -9,8 +9,8 @@
 //           chosen so that the whole grid is about one resident wave (4 CTAs of 256 threads per SM);
 //   loop  : a thread visits its columns in ascending order, four 16-byte vectors (bf16x8 / f32x4) per
 //           iteration, the next four already in flight (register double buffer), and keeps a running
-//           (max, S, T) with S = sum 2^d, T = sum 2^d * d, d = x*log2(e) - base: one FMA, one ex2.approx,
-//           one add and one FMA per element.  The base follows the maximum lazily: it moves, and S and T
+//           (max, S, T) with S = sum 2^d, T = sum 2^d * d, d = x*log2(e) - base: one ex2.approx per element
+//           and one packed fp32x2 FMA, add and FMA per pair of elements.  The base follows the maximum lazily: it moves, and S and T
 //           are rescaled (S' = 2^dl S, T' = 2^dl (T + dl S), dl = old base - new base), only when a value
 //           exceeds it by more than 2^64, so the common path has no data-dependent branch.  Logits are
 //           clamped from below at -1e38 (packed bf16 max on the raw words), which keeps d finite:
@@ -67,6 +67,31 @@ __device__ __forceinline__ Partial merge(Partial a, Partial b) {
     return hi;
 }
 
+// ticket: release (the partial written just before by this thread is visible to whoever sees the count) and
+// acquire (whoever completes the count sees every earlier partial)
+__device__ __forceinline__ int ticket_add(int* addr, int v) {
+    int old;
+    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+    return old;
+}
+// packed pairs of fp32 (one 64-bit register): two lanes per FMA / add issue slot
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ unsigned int max_bf16x2(unsigned int a, unsigned int b) {
@@ -104,6 +129,11 @@ struct Loader<__nv_bfloat16> {
             x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
     }
+    static __device__ __forceinline__ void widen2(const uint4& u, f32x2 (&x)[4]) {
+        const unsigned int w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+    }
     static __device__ __forceinline__ float one(const __nv_bfloat16* p) {
         return fmaxf(__bfloat162float(*p), __uint_as_float(kXMinF32));
     }
@@ -129,6 +159,10 @@ struct Loader<float> {
     static __device__ __forceinline__ void widen(const uint4& u, float (&x)[4]) {
         x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y);
         x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
+    }
+    static __device__ __forceinline__ void widen2(const uint4& u, f32x2 (&x)[2]) {
+        x[0] = pack2(__uint_as_float(u.x), __uint_as_float(u.y));
+        x[1] = pack2(__uint_as_float(u.z), __uint_as_float(u.w));
     }
     static __device__ __forceinline__ float one(const float* p) { return fmaxf(*p, __uint_as_float(kXMinF32)); }
 };
@@ -200,26 +234,23 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     pdl_wait();                 // the previous kernel of the stream has completed: the logits are final
     pdl_launch_dependents();
 
-    float m = -INFINITY, base = base_of(-INFINITY), S = 0.f, Tt = 0.f;
+    // running state: maximum, exponent base, and S, T as two packed lanes each
+    float m = -INFINITY, base = base_of(-INFINITY);
+    f32x2 S2 = pack2(0.f, 0.f), T2 = pack2(0.f, 0.f);
     int mcol = -1, mspan = 0;   // where the maximum was raised: first column of the vectors to look at again, and how many
-    auto accumulate = [&](const float (&x)[EPV]) {
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-            const float d = fmaf(x[i], kLog2e, -base);
-            const float e = fast_exp2(d);
-            S += e;
-            Tt = fmaf(e, d, Tt);
-        }
-    };
+    const f32x2 kL2 = pack2(kLog2e, kLog2e);
     auto rebase_if_needed = [&](float vmax) {
         if (fmaf(vmax, kLog2e, -base) > kRebase) {   // rare
             const float nb = base_of(vmax);
-            if (S > 0.f) {
-                const float dl = fmaxf(base - nb, kDClamp);
-                const float c = fast_exp2(dl);
-                Tt = c * fmaf(dl, S, Tt);
-                S *= c;
-            }
+            const float dl = fmaxf(base - nb, kDClamp);
+            const float c = fast_exp2(dl);
+            float s0, s1, t0, t1;
+            unpack2(S2, s0, s1);
+            unpack2(T2, t0, t1);
+            t0 = s0 > 0.f ? c * fmaf(dl, s0, t0) : 0.f;
+            t1 = s1 > 0.f ? c * fmaf(dl, s1, t1) : 0.f;
+            S2 = pack2(s0 * c, s1 * c);
+            T2 = pack2(t0, t1);
             base = nb;
         }
     };
@@ -255,11 +286,20 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
             m = up ? it_max : m;
             mcol = up ? col0 : mcol;
             mspan = up ? kUnroll : mspan;
+            const f32x2 nb2 = pack2(-base, -base);
 #pragma unroll
             for (int v = 0; v < kUnroll; ++v) {
-                float x[EPV];
-                Loader<T>::widen(raw[v], x);
-                accumulate(x);
+                f32x2 x2[EPV / 2];
+                Loader<T>::widen2(raw[v], x2);
+#pragma unroll
+                for (int i = 0; i < EPV / 2; ++i) {
+                    const f32x2 d2 = fma2(x2[i], kL2, nb2);
+                    float d0, d1;
+                    unpack2(d2, d0, d1);
+                    const f32x2 e2 = pack2(fast_exp2(d0), fast_exp2(d1));
+                    S2 = add2(S2, e2);
+                    T2 = fma2(e2, d2, T2);
+                }
             }
         } else {
 #pragma unroll
@@ -282,13 +322,18 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                 m = up ? vmax : m;
                 mcol = up ? col : mcol;
                 mspan = up ? 1 : mspan;
+                float s0, s1, t0, t1;
+                unpack2(S2, s0, s1);
+                unpack2(T2, t0, t1);
 #pragma unroll
                 for (int i = 0; i < EPV; ++i) {   // 2^-inf = 0, and that product is kept out of T
                     const float d = fmaf(x[i], kLog2e, -base);
                     const float e = fast_exp2(d);
-                    S += e;
-                    Tt = (x[i] == -INFINITY) ? Tt : fmaf(e, d, Tt);
+                    s0 += e;
+                    t0 = (x[i] == -INFINITY) ? t0 : fmaf(e, d, t0);
                 }
+                S2 = pack2(s0, s1);
+                T2 = pack2(t0, t1);
             }
         }
     };
@@ -306,6 +351,15 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     }
 
     // ---- CTA-wide maximum; the threads that attained it find its first column ---------------------------
+    // every thread asks again for the vectors that raised its maximum (L2 hits, in flight during the reduction);
+    // only the threads that attained the CTA's maximum will look at them
+    uint4 again[kUnroll];
+#pragma unroll
+    for (int v = 0; v < kUnroll; ++v) {
+        again[v] = make_uint4(0u, 0u, 0u, 0u);
+        const int col = mcol + v * kVStride;
+        if (v < mspan && mcol >= 0 && col + EPV <= c_end) again[v] = __ldg(reinterpret_cast<const uint4*>(rowp + col));
+    }
     float wm = m;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
@@ -316,14 +370,33 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     for (int w = 1; w < kGateThreads / 32; ++w) M = fmaxf(M, s_m[w]);
     int idx = 0x7fffffff;
     if (m == M && mcol >= 0) {
-        for (int v = mspan - 1; v >= 0; --v) {   // descending: the smallest column survives
-            const int col = mcol + v * kVStride;
 #pragma unroll
-            for (int i = EPV - 1; i >= 0; --i)
-                if (col + i < c_end && Loader<T>::one(rowp + col + i) == M) idx = col + i;
+        for (int v = kUnroll - 1; v >= 0; --v) {   // descending: the smallest column survives
+            const int col = mcol + v * kVStride;
+            if (v >= mspan) continue;
+            if (col + EPV <= c_end) {
+                float x[EPV];
+                Loader<T>::clamp(again[v]);
+                Loader<T>::widen(again[v], x);
+#pragma unroll
+                for (int i = EPV - 1; i >= 0; --i)
+                    if (x[i] == M) idx = col + i;
+            } else {   // the chunk's ragged last vector
+#pragma unroll
+                for (int i = EPV - 1; i >= 0; --i)
+                    if (col + i < c_end && Loader<T>::one(rowp + col + i) == M) idx = col + i;
+            }
         }
     }
     // ---- sums against the CTA's base, first column of the maximum --------------------------------------
+    float S, Tt;
+    {
+        float s0, s1, t0, t1;
+        unpack2(S2, s0, s1);
+        unpack2(T2, t0, t1);
+        S = s0 + s1;
+        Tt = t0 + t1;
+    }
     if (S > 0.f) {
         const float dl = fmaxf(base - base_of(M), kDClamp);
         const float c = fast_exp2(dl);
@@ -348,17 +421,15 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
         for (int w = 0; w < kGateThreads / 32; ++w) { Ss += s_S[w]; Ts += s_T[w]; Midx = min(Midx, s_i[w]); }
         *reinterpret_cast<float4*>(&p.partials[(long long)row * p.splits + split]) =
             make_float4(M, Ss, Ts, __int_as_float(Midx));
-        __threadfence();
         int last;
         if (p.single_level)
-            last = (atomicAdd(&p.seq_ticket[seq], 1) == p.rows_per_seq * p.splits - 1);
+            last = (ticket_add(&p.seq_ticket[seq], 1) == p.rows_per_seq * p.splits - 1);
         else
-            last = (atomicAdd(&p.row_ticket[row], 1) == p.splits - 1);
+            last = (ticket_add(&p.row_ticket[row], 1) == p.splits - 1);
         s_last = last;
     }
-    __syncthreads();
+    __syncthreads();   // orders the ticket's acquire before the other threads' reads of the partials
     if (!s_last) return;
-    __threadfence();
 
     if (p.single_level) {
         // ---- last CTA of the sequence: finish every row, then the masked maximum and the decision ----
@@ -421,12 +492,10 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     int seq_last = 0;
     if (lane == 0) {
         p.row_ticket[row] = 0;
-        __threadfence();
-        seq_last = (atomicAdd(&p.seq_ticket[seq], 1) == p.rows_per_seq - 1);
+        seq_last = (ticket_add(&p.seq_ticket[seq], 1) == p.rows_per_seq - 1);
     }
     seq_last = __shfl_sync(0xffffffffu, seq_last, 0);
     if (!seq_last) return;
-    __threadfence();
     float E = -INFINITY;
     for (int r = lane; r < p.rows_per_seq; r += 32) {
         const int rr = seq * p.rows_per_seq + r;
@@ -467,8 +536,7 @@ void plan_chunks(int n_rows, int vocab, int* splits, int* chunk) {
     long long per = (vocab + want - 1) / want;
     const long long per_min = (vocab + kMaxSplits - 1) / kMaxSplits;
     if (per < per_min) per = per_min;
-    const long long step = (long long)kUnroll * slab;   // one loop iteration of the bf16 kernel
-    per = per >= 2 * step ? (per + step - 1) / step * step : (per + slab - 1) / slab * slab;
+    per = (per + slab - 1) / slab * slab;
     *chunk = (int)per;
     *splits = (int)((vocab + per - 1) / per);
 }
