@@ -132,6 +132,7 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     a.scale = desc->scale > 0.f ? desc->scale : 1.0f / sqrtf((float)desc->head_dim);
     const cudaError_t e = fused                  ? launch_attend_skip(a, k_new, v_new, active_idx, s)
                           : desc->dtype != EC_BF16 ? launch_attend_f32(a, s)
+                          : (use_tc(*desc) && forced_impl() != 2 && attend_dense_supported(*desc, n_active)) ? launch_attend_dense(a, s)
                           : use_tc(*desc)        ? launch_attend_bf16_tc(a, s)
                                                  : launch_attend_bf16(a, s);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;

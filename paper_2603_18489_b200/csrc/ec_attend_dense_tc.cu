@@ -1,0 +1,370 @@
+// ec_attend, recompute step and other dense cases (bf16, head_dim 128, more than 256 packed query rows per
+// kv head): bidirectional attention of every active row over the whole cache on the Blackwell tensor cores
+// (Appendix A of the paper, full branch; Algorithm 1 FullPrefill / FullRecompute).
+//
+// The step is bound by the tensor pipe and, next to it, by the exponentials of the softmax.  One CTA owns
+// TWO 128-row tiles of the packed (active row x query heads of one kv head) axis and walks over all
+// 128-key tiles of that kv head; while the softmax of one row tile runs, the tensor core works for the other.
+//   warp 0      TMA producer: K and V tiles ([128 keys x 128] bf16, one 4-D box each: [2 halves][128 keys]
+//               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...);
+//   warp 1      tcgen05.mma issuer (one thread): S_t = Q_t K^T (both operands K-major in shared memory) into
+//               the TMEM columns of row tile t, and O_t += P_t V with P_t read from TENSOR MEMORY (it
+//               overwrites the first 64 columns of S_t as packed bf16) and V MN-major from shared memory.
+//               Order per key tile j:  P V_0(j), S_0(j+1), P V_1(j), S_1(j+1): the pipe executes in order,
+//               so S_t(j+1) cannot overwrite P_t(j) before P V_t(j) has read it;
+//   warps 2..5  softmax of row tile 0, warps 6..9 of row tile 1: thread = query row = TMEM lane; tcgen05.ld of
+//               the 128 scores, running max / sum, exp2 with the scale folded in (packed fp32x2 FMA), P
+//               rounded to bf16 and stored back with tcgen05.st; the O accumulator is only rescaled when a
+//               row maximum grows by more than 2^8 (the stale maximum stays the reference otherwise).
+// TMEM (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,384), O_1 [384,512).
+// Shared memory: Q_0, Q_1 (32 KB each, staged once), five 32 KB K/V slots, barriers: 225 KB, one CTA per SM.
+// Every mbarrier wait is bounded; a wait that runs out sets EC_ERR_TIMEOUT in the caller's dev_status word and
+// a CTA-wide abort flag that makes all later waits fall through; the CTA still frees its TMEM and exits.
+#include "ec_common.cuh"
+#include "ec_tc_ptx.cuh"
+
+namespace ec {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 128, HD = 128;
+constexpr int kThreads = 64 + 2 * 128;
+constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
+constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
+constexpr int kSlots = 5;
+constexpr uint32_t OFF_Q = 0;              // two tiles
+constexpr uint32_t OFF_RING = 2 * TILE;
+constexpr uint32_t OFF_BAR = OFF_RING + kSlots * TILE;   // 224 KB
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 256 + 1024;    // + barrier block + alignment slack
+constexpr uint32_t TM_COLS = 512;
+constexpr uint32_t TM_S = 0, TM_O = 256;   // + 128 * tile
+
+enum { B_FULL = 0, B_EMPTY = kSlots, B_SFULL = 2 * kSlots, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 2,
+       B_QFULL = B_PVDONE + 2, B_COUNT = B_QFULL + 1 };
+
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+struct DenseParams {
+    const __nv_bfloat16* q;
+    __nv_bfloat16* out;
+    int32_t* dev_status;
+    int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
+    float scale_log2;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const DenseParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (s2u(smem_raw) + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - s2u(smem_raw));
+    const uint32_t bars = base + OFF_BAR;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + OFF_BAR + B_COUNT * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + OFF_BAR + B_COUNT * 8 + 4);
+    auto bar = [&](int idx) { return bars + idx * 8; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int pair = blockIdx.x, bh = blockIdx.y;
+    const int b = bh / p.n_kv_heads, hk = bh % p.n_kv_heads;
+    const int r_pair = pair * 2 * BM;
+    const int n_tiles_q = (p.rows_total - r_pair > BM) ? 2 : 1;   // row tiles of this CTA that hold rows
+    const int T = (p.ctx_len + BN - 1) / BN;
+
+    if (tid == 0) {
+        prefetch_map(&map_k);
+        prefetch_map(&map_v);
+        for (int i = 0; i < B_COUNT; ++i)
+            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 128u : (i == B_QFULL ? 256u : 1u));
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(tmem_slot)), "r"(TM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        fence_before();
+    }
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = *tmem_slot;
+    pdl_wait();   // the previous kernel of the stream has completed; global memory may be touched
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        // ================================ TMA producer ======================================
+        if (lane == 0) {
+            for (int n = 0; n < 2 * T; ++n) {   // ring index: K_j = 2j, V_j = 2j + 1
+                const int slot = n % kSlots, u = n / kSlots;
+                if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
+                mbar_expect_tx(bar(B_FULL + slot), TILE);
+                tma_load_4d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, bh, bar(B_FULL + slot));
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ========================================
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = instr_desc(BN, 0), IDESC_PV = instr_desc(HD, 1);
+            auto wait_full = [&](int n) { mbar_wait(bar(B_FULL + n % kSlots), (n / kSlots) & 1, abort_flag, p.dev_status); };
+            auto issue_s = [&](int t, int j) {
+                const uint32_t kst = base + OFF_RING + ((2 * j) % kSlots) * TILE;
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k) {
+                    const uint32_t koff = (k >> 2) * SUB + (k & 3) * 32;
+                    mma_ss(tmem + TM_S + t * 128, smem_desc(base + OFF_Q + t * TILE + koff, 16, 1024),
+                           smem_desc(kst + koff, 16, 1024), IDESC_S, k > 0);
+                }
+                commit(bar(B_SFULL + t));
+            };
+            mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
+            wait_full(0);
+            fence_after();
+            for (int t = 0; t < n_tiles_q; ++t) issue_s(t, 0);
+            commit(bar(B_EMPTY + 0));   // K_0 is free once both S(0) have run
+            for (int j = 0; j < T; ++j) {
+                wait_full(2 * j + 1);   // V_j
+                if (j + 1 < T) wait_full(2 * j + 2);   // K_{j+1}
+                const uint32_t vst = base + OFF_RING + ((2 * j + 1) % kSlots) * TILE;
+                for (int t = 0; t < n_tiles_q; ++t) {
+                    mbar_wait(bar(B_PFULL + t), j & 1, abort_flag, p.dev_status);
+                    fence_after();
+#pragma unroll
+                    for (int k = 0; k < BN / 16; ++k)
+                        mma_ts(tmem + TM_O + t * 128, tmem + TM_S + t * 128 + k * 8, smem_desc(vst + k * 2048, SUB, 1024),
+                               IDESC_PV, (j > 0 || k > 0));
+                    commit(bar(B_PVDONE + t));
+                    if (j + 1 < T) issue_s(t, j + 1);
+                }
+                commit(bar(B_EMPTY + (2 * j + 1) % kSlots));              // V_j
+                if (j + 1 < T) commit(bar(B_EMPTY + (2 * j + 2) % kSlots));   // K_{j+1}
+            }
+        }
+    } else {
+        // ====================== Q staging, then softmax (warps 2..9) =========================
+        const int stid = tid - 64;
+        // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
+        for (int c = stid; c < 2 * BM * (HD / 8); c += 2 * BM) {
+            const int row = c >> 4, ch = c & 15;   // row in [0, 256)
+            const int r = r_pair + row;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (r < p.rows_total) {
+                const int i = r / p.group, j = r % p.group;
+                v = __ldg(reinterpret_cast<const uint4*>(
+                    p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + j) * HD + ch * 8));
+            }
+            const int t = row >> 7, rt = row & 127;
+            const uint32_t off = OFF_Q + t * TILE + (ch >> 3) * SUB + (rt >> 3) * 1024 + (rt & 7) * 128 + (((ch & 7) ^ (rt & 7)) << 4);
+            *reinterpret_cast<uint4*>(gbase + off) = v;
+        }
+        fence_async_smem();   // generic-proxy writes of Q -> visible to the tensor core (async proxy)
+        mbar_arrive(bar(B_QFULL));
+
+        const int t = (warp - 2) >> 2;              // row tile of this warp
+        const int quarter = warp & 3;               // TMEM lanes this warp may touch
+        const int row = quarter * 32 + lane;        // row of the tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const uint32_t tm_s = tmem + lane_addr + TM_S + t * 128;
+        const uint32_t tm_o = tmem + lane_addr + TM_O + t * 128;
+        const int r = r_pair + t * BM + row;
+        if (t < n_tiles_q) {
+            float m_used = -INFINITY, l_run = 0.f;
+            const float sl2 = p.scale_log2;
+            const f32x2 sl2_2 = pk(sl2, sl2);
+            for (int j = 0; j < T; ++j) {
+                mbar_wait(bar(B_SFULL + t), j & 1, abort_flag, p.dev_status);
+                fence_after();
+                uint32_t sr[BN];
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c) ld32(tm_s + c * 32, sr + c * 32);
+                wait_ld();
+                const int key0 = j * BN;
+                if (key0 + BN > p.ctx_len) {
+#pragma unroll
+                    for (int c = 0; c < BN; ++c)
+                        if (key0 + c >= p.ctx_len) sr[c] = 0xff800000u;   // -inf
+                }
+                float mx[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sr[c]);
+#pragma unroll
+                for (int c = 8; c < BN; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sr[c]));
+                const float mrow = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_tile = mrow * sl2;
+                float factor = 1.f;
+                if (m_tile > m_used + 8.f || m_used == -INFINITY) {   // stale maximum allowed up to 2^8
+                    factor = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_tile);
+                    m_used = m_tile;
+                }
+                const bool need_rescale = (j > 0) && __any_sync(0xffffffffu, factor != 1.f);
+                const f32x2 mneg2 = pk(-m_used, -m_used);
+                f32x2 sum2[2] = {pk(0.f, 0.f), pk(0.f, 0.f)};
+                uint32_t pw[BN / 2];
+#pragma unroll
+                for (int c = 0; c < BN / 2; ++c) {
+                    const f32x2 d2 = fma2(pk(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sl2_2, mneg2);
+                    float d0, d1;
+                    upk(d2, d0, d1);
+                    const float e0 = fast_exp2(d0), e1 = fast_exp2(d1);
+                    sum2[c & 1] = add2(sum2[c & 1], pk(e0, e1));
+                    pw[c] = pack_bf16x2(e0, e1);
+                }
+                {
+                    float a0, a1, b0, b1;
+                    upk(sum2[0], a0, a1);
+                    upk(sum2[1], b0, b1);
+                    l_run = fmaf(l_run, factor, (a0 + a1) + (b0 + b1));
+                }
+                if (need_rescale) {
+                    // O holds tiles < j: P V of tile j - 1 must have completed before this row's accumulator is scaled
+                    mbar_wait(bar(B_PVDONE + t), (j - 1) & 1, abort_flag, p.dev_status);
+                    fence_after();
+#pragma unroll
+                    for (int c = 0; c < HD / 32; ++c) {
+                        uint32_t o[32];
+                        ld32(tm_o + c * 32, o);
+                        wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        st32(tm_o + c * 32, o);
+                    }
+                }
+                // P (bf16 pairs) over the first 64 columns of S_t
+                st32(tm_s, pw);
+                st32(tm_s + 32, pw + 32);
+                wait_st();
+                fence_before();
+                mbar_arrive(bar(B_PFULL + t));
+            }
+
+            // ---- epilogue: normalise and store -------------------------------------------------
+            mbar_wait(bar(B_PVDONE + t), (T - 1) & 1, abort_flag, p.dev_status);
+            fence_after();
+            const bool valid = r < p.rows_total;
+            const int i = valid ? r / p.group : 0, jh = valid ? r % p.group : 0;
+            __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD;
+            const float inv = 1.f / l_run;
+#pragma unroll
+            for (int c = 0; c < HD / 32; ++c) {
+                uint32_t o[32];
+                ld32(tm_o + c * 32, o);
+                wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
+                    }
+                }
+            }
+        }
+        fence_before();
+    }
+
+    __syncthreads();
+    if (warp == 1) {
+        fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// cache [B*Hkv, L, 128] bf16 seen as 4-D {64 columns, key, half, head}: one box {64, 128, 2, 1} lands as
+// [half][key][64 columns], the two 128-byte-swizzled halves of a [128 keys x 128] tile; keys beyond L read as zero
+bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {64, (cuuint64_t)ctx_len, 2, (cuuint64_t)bh};
+    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)ctx_len * HD * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)BN, 2, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(cache), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// the two-tile kernel has no key split: it is used when the (row-tile pair, kv head) units fill the GPU
+bool attend_dense_supported(const ec_attn_desc& d, int n_active) {
+    if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
+    const long long rows = (long long)n_active * (d.n_q_heads / d.n_kv_heads);
+    const long long pairs = (rows + 2 * BM - 1) / (2 * BM);
+    const long long bh = (long long)d.batch * d.n_kv_heads;
+    if (bh > 65535 || pairs > 0x7fffffffLL) return false;
+    return pairs * bh >= sm_count() / 2;
+}
+
+cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
+    const int bh = a.d.batch * a.d.n_kv_heads;
+    CUtensorMap map_k, map_v;
+    if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
+        return cudaErrorInvalidValue;
+    DenseParams p;
+    p.q = static_cast<const __nv_bfloat16*>(a.q);
+    p.out = static_cast<__nv_bfloat16*>(a.out);
+    p.dev_status = a.dev_status;
+    p.n_active = a.n_active;
+    p.ctx_len = a.d.ctx_len;
+    p.n_q_heads = a.d.n_q_heads;
+    p.n_kv_heads = a.d.n_kv_heads;
+    p.group = a.d.n_q_heads / a.d.n_kv_heads;
+    p.rows_total = a.n_active * p.group;
+    p.scale_log2 = a.scale * kLog2e;
+    static bool attr_done[64] = {};   // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(attend_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((p.rows_total + 2 * BM - 1) / (2 * BM), bh, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attend_dense_kernel, map_k, map_v, p);
+}
+
+}  // namespace ec

@@ -73,6 +73,9 @@ cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);      /
 bool attend_skip_supported(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                cudaStream_t stream);
+// two-row-tile dense path (bf16, head_dim 128): used when its (row-tile pair, kv head) units fill the GPU
+bool attend_dense_supported(const ec_attn_desc& d, int n_active);
+cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream);
 size_t attend_tc_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_bf16_tc(const AttendArgs& a, cudaStream_t stream);   // tcgen05 path (head_dim 128)
 
