@@ -12,10 +12,14 @@
 //               overwrites the first 64 columns of S_t as packed bf16) and V MN-major from shared memory.
 //               Order per key tile j:  P V_0(j), S_0(j+1), P V_1(j), S_1(j+1): the pipe executes in order,
 //               so S_t(j+1) cannot overwrite P_t(j) before P V_t(j) has read it;
-//   warps 2..5  softmax of row tile 0, warps 6..9 of row tile 1: thread = query row = TMEM lane; tcgen05.ld of
-//               the 128 scores, running max / sum, exp2 with the scale folded in (packed fp32x2 FMA), P
-//               rounded to bf16 and stored back with tcgen05.st; the O accumulator is only rescaled when a
-//               row maximum grows by more than 2^8 (the stale maximum stays the reference otherwise).
+//   warps 2..17 softmax, four warpgroups: (row tile 0 / 1) x (keys 0..63 / 64..127 of the tile).  A query row
+//               (= TMEM lane) is shared by two threads in warps that own the same lanes; they exchange
+//               their half-row maxima through shared memory (a 64-thread named barrier), then each does
+//               tcgen05.ld of its 64 scores, exp2 with the scale folded in (packed fp32x2 FMA), its share of
+//               the row sum, P rounded to bf16 and stored back with tcgen05.st; the O accumulator is only
+//               rescaled when a row maximum grows by more than 2^8 (the stale maximum stays the reference
+//               otherwise).  Halving the per-thread row shortens the softmax that sits between two uses of
+//               the tensor pipe for the same row tile.
 // TMEM (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,384), O_1 [384,512).
 // Shared memory: Q_0, Q_1 (32 KB each, staged once), five 32 KB K/V slots, barriers: 225 KB, one CTA per SM.
 // Every mbarrier wait is bounded; a wait that runs out sets EC_ERR_TIMEOUT in the caller's dev_status word and
@@ -29,14 +33,18 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 128, HD = 128;
-constexpr int kThreads = 64 + 2 * 128;
+constexpr int kSoftThreads = 512;          // four softmax warpgroups: (row tile) x (64-column half)
+constexpr int kThreads = 64 + kSoftThreads;
+constexpr int kPolyOf5 = 0;                // pairs out of every five whose exponentials go to the FMA pipe
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr int kSlots = 5;
 constexpr uint32_t OFF_Q = 0;              // two tiles
 constexpr uint32_t OFF_RING = 2 * TILE;
 constexpr uint32_t OFF_BAR = OFF_RING + kSlots * TILE;   // 224 KB
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256 + 1024;    // + barrier block + alignment slack
+constexpr uint32_t OFF_XCH = OFF_BAR + 256;               // [2 tiles][2 halves][128 rows] floats
+constexpr uint32_t SMEM_BYTES = 232448;                   // all of a CTA's 227 KB; the rest is alignment slack
+constexpr uint32_t SMEM_NEEDED = OFF_XCH + 2 * 2 * BM * 4;
 constexpr uint32_t TM_COLS = 512;
 constexpr uint32_t TM_S = 0, TM_O = 256;   // + 128 * tile
 
@@ -61,6 +69,36 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
     return r;
 }
 
+__device__ __forceinline__ void named_barrier(int id, int n_threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// 2^x for a pair of values on the FMA pipe (the MUFU pipe is the softmax's bottleneck, so a share of the
+// exponentials is computed here instead): x = n + f with n = round(x), |f| <= 1/2, 2^f by a cubic fitted for a
+// maximum relative error of 7.5e-5 (far below the bf16 rounding of P), and n added to the exponent field.
+// Inputs below -126 give (flushed) zero.
+__device__ __forceinline__ void exp2_poly2(f32x2 d2, float& e0, float& e1) {
+    float x0, x1;
+    upk(d2, x0, x1);
+    const f32x2 x2 = pk(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const f32x2 magic2 = pk(12582912.f, 12582912.f);   // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+    const f32x2 t2 = add2(x2, magic2);
+    const f32x2 n2 = add2(t2, pk(-12582912.f, -12582912.f));
+    const f32x2 f2 = fma2(n2, pk(-1.f, -1.f), x2);
+    f32x2 p2 = fma2(f2, pk(0.05517146f, 0.05517146f), pk(0.24261086f, 0.24261086f));
+    p2 = fma2(p2, f2, pk(0.69326097f, 0.69326097f));
+    p2 = fma2(p2, f2, pk(0.9999281f, 0.9999281f));
+    float p0, p1, t0, t1;
+    upk(p2, p0, p1);
+    upk(t2, t0, t1);
+    e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
 struct DenseParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
@@ -77,7 +115,12 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const uint32_t bars = base + OFF_BAR;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + OFF_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + OFF_BAR + B_COUNT * 8 + 4);
+    float* xch = reinterpret_cast<float*>(gbase + OFF_XCH);
     auto bar = [&](int idx) { return bars + idx * 8; };
+    if (base - s2u(smem_raw) + SMEM_NEEDED > SMEM_BYTES) {   // never with the 1024-byte alignment the runtime gives
+        if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, (int)EC_ERR_CUDA);
+        return;
+    }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int pair = blockIdx.x, bh = blockIdx.y;
@@ -90,7 +133,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         prefetch_map(&map_k);
         prefetch_map(&map_v);
         for (int i = 0; i < B_COUNT; ++i)
-            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 128u : (i == B_QFULL ? 256u : 1u));
+            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 256u : (i == B_QFULL ? (uint32_t)kSoftThreads : 1u));
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -155,10 +198,10 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
         }
     } else {
-        // ====================== Q staging, then softmax (warps 2..9) =========================
+        // ====================== Q staging, then softmax (warps 2..17) ========================
         const int stid = tid - 64;
         // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
-        for (int c = stid; c < 2 * BM * (HD / 8); c += 2 * BM) {
+        for (int c = stid; c < 2 * BM * (HD / 8); c += kSoftThreads) {
             const int row = c >> 4, ch = c & 15;   // row in [0, 256)
             const int r = r_pair + row;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -174,13 +217,19 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         fence_async_smem();   // generic-proxy writes of Q -> visible to the tensor core (async proxy)
         mbar_arrive(bar(B_QFULL));
 
-        const int t = (warp - 2) >> 2;              // row tile of this warp
-        const int quarter = warp & 3;               // TMEM lanes this warp may touch
+        // A row of a tile is shared by two threads, one per 64-column half, in warps that own the same TMEM
+        // lanes: softmax warp ws = warp - 2 -> row tile ws / 8, column half (ws / 4) % 2, lanes 32 * (warp % 4).
+        const int ws = warp - 2;
+        const int t = ws >> 3, h = (ws >> 2) & 1;
+        const int quarter = warp & 3;
         const int row = quarter * 32 + lane;        // row of the tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t tm_s = tmem + lane_addr + TM_S + t * 128;
         const uint32_t tm_o = tmem + lane_addr + TM_O + t * 128;
         const int r = r_pair + t * BM + row;
+        float* xch_mine = xch + (t * 2 + h) * BM + row;        // exchanged with the partner thread of the row
+        const float* xch_other = xch + (t * 2 + (1 - h)) * BM + row;
+        const int pair_bar = 1 + t * 4 + quarter;              // named barrier of the two warps that share these rows
         if (t < n_tiles_q) {
             float m_used = -INFINITY, l_run = 0.f;
             const float sl2 = p.scale_log2;
@@ -188,23 +237,25 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             for (int j = 0; j < T; ++j) {
                 mbar_wait(bar(B_SFULL + t), j & 1, abort_flag, p.dev_status);
                 fence_after();
-                uint32_t sr[BN];
-#pragma unroll
-                for (int c = 0; c < BN / 32; ++c) ld32(tm_s + c * 32, sr + c * 32);
+                uint32_t sr[BN / 2];
+                ld32(tm_s + h * 64, sr);
+                ld32(tm_s + h * 64 + 32, sr + 32);
                 wait_ld();
-                const int key0 = j * BN;
-                if (key0 + BN > p.ctx_len) {
+                const int key0 = j * BN + h * 64;
+                if (key0 + 64 > p.ctx_len) {
 #pragma unroll
-                    for (int c = 0; c < BN; ++c)
+                    for (int c = 0; c < 64; ++c)
                         if (key0 + c >= p.ctx_len) sr[c] = 0xff800000u;   // -inf
                 }
-                float mx[8];
+                float mx[4];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sr[c]);
+                for (int c = 0; c < 4; ++c) mx[c] = __uint_as_float(sr[c]);
 #pragma unroll
-                for (int c = 8; c < BN; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sr[c]));
-                const float mrow = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                const float m_tile = mrow * sl2;
+                for (int c = 4; c < 64; c += 2) mx[(c >> 1) & 3] = max3(mx[(c >> 1) & 3], __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+                const float mloc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                *xch_mine = mloc;
+                named_barrier(pair_bar, 64);   // both halves of the row have loaded their scores and posted their maxima
+                const float m_tile = fmaxf(mloc, *xch_other) * sl2;
                 float factor = 1.f;
                 if (m_tile > m_used + 8.f || m_used == -INFINITY) {   // stale maximum allowed up to 2^8
                     factor = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_tile);
@@ -213,13 +264,19 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const bool need_rescale = (j > 0) && __any_sync(0xffffffffu, factor != 1.f);
                 const f32x2 mneg2 = pk(-m_used, -m_used);
                 f32x2 sum2[2] = {pk(0.f, 0.f), pk(0.f, 0.f)};
-                uint32_t pw[BN / 2];
+                uint32_t pw[32];
 #pragma unroll
-                for (int c = 0; c < BN / 2; ++c) {
+                for (int c = 0; c < 32; ++c) {
                     const f32x2 d2 = fma2(pk(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sl2_2, mneg2);
-                    float d0, d1;
-                    upk(d2, d0, d1);
-                    const float e0 = fast_exp2(d0), e1 = fast_exp2(d1);
+                    float e0, e1;
+                    if (kPolyOf5 > 0 && c % 5 < kPolyOf5) {   // this share of the pairs on the FMA pipe, the rest on the MUFU pipe
+                        exp2_poly2(d2, e0, e1);
+                    } else {
+                        float d0, d1;
+                        upk(d2, d0, d1);
+                        e0 = fast_exp2(d0);
+                        e1 = fast_exp2(d1);
+                    }
                     sum2[c & 1] = add2(sum2[c & 1], pk(e0, e1));
                     pw[c] = pack_bf16x2(e0, e1);
                 }
@@ -227,41 +284,43 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     float a0, a1, b0, b1;
                     upk(sum2[0], a0, a1);
                     upk(sum2[1], b0, b1);
-                    l_run = fmaf(l_run, factor, (a0 + a1) + (b0 + b1));
+                    l_run = fmaf(l_run, factor, (a0 + a1) + (b0 + b1));   // this half's share of the row sum
                 }
                 if (need_rescale) {
-                    // O holds tiles < j: P V of tile j - 1 must have completed before this row's accumulator is scaled
+                    // O holds tiles < j: P V of tile j - 1 must have completed before the accumulator is scaled;
+                    // each of the two threads of a row scales its 64 columns
                     mbar_wait(bar(B_PVDONE + t), (j - 1) & 1, abort_flag, p.dev_status);
                     fence_after();
 #pragma unroll
-                    for (int c = 0; c < HD / 32; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
-                        ld32(tm_o + c * 32, o);
+                        ld32(tm_o + h * 64 + c * 32, o);
                         wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                        st32(tm_o + c * 32, o);
+                        st32(tm_o + h * 64 + c * 32, o);
                     }
                 }
-                // P (bf16 pairs) over the first 64 columns of S_t
-                st32(tm_s, pw);
-                st32(tm_s + 32, pw + 32);
+                // P (bf16 pairs) over the first 64 columns of S_t: this thread's 64 keys are columns [32 h, 32 h + 32)
+                st32(tm_s + h * 32, pw);
                 wait_st();
                 fence_before();
                 mbar_arrive(bar(B_PFULL + t));
             }
 
-            // ---- epilogue: normalise and store -------------------------------------------------
+            // ---- epilogue: normalise and store this thread's 64 columns ---------------------------
             mbar_wait(bar(B_PVDONE + t), (T - 1) & 1, abort_flag, p.dev_status);
             fence_after();
+            *xch_mine = l_run;
+            named_barrier(pair_bar, 64);
+            const float inv = 1.f / (l_run + *xch_other);
             const bool valid = r < p.rows_total;
             const int i = valid ? r / p.group : 0, jh = valid ? r % p.group : 0;
-            __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD;
-            const float inv = 1.f / l_run;
+            __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + h * 64;
 #pragma unroll
-            for (int c = 0; c < HD / 32; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t o[32];
-                ld32(tm_o + c * 32, o);
+                ld32(tm_o + h * 64 + c * 32, o);
                 wait_ld();
                 if (valid) {
 #pragma unroll
