@@ -40,6 +40,35 @@ L2_BYTES = 126 * 1024 * 1024
 DEFAULT_WORKLOAD = "c2_llada_l768"
 
 
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/.  A figure is reported only while the kernel's source file still has the hash it had when the
+# counters were taken; after any change to the kernel it reads null until the capture is redone.
+NCU_TRAFFIC = {
+    "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
+                    "sha256": "33bdbd0bbaf1065a8524d965ba870f214f2555de4dc95aa6cd23f979c5b9fcdb",
+                    "bytes_per_launch": {"c2_llada_l768": 12930816, "c5_llada_l4096": 68199168}},
+    "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
+                     "sha256": "8b9b93fb78eb526dd48d92e6b73050e6a46dcac25c98baaf4c4c32f7162da1d1",
+                     "bytes_per_launch": {"c4_llada_l2048": 51188992, "c5_llada_l4096": 116217856}},
+    "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
+                     "sha256": "f7350fa75a2ea8d82120fbfb3ea587e366e2a8716e4a2a11e71f8f323e1ef9f3",
+                     "bytes_per_launch": {"c5_llada_l4096_b8": 65324032}},
+}
+
+
+def _ncu_traffic(kernel: str, workload: str):
+    import hashlib
+
+    e = NCU_TRAFFIC[kernel]
+    try:
+        h = hashlib.sha256(open(os.path.join(ROOT, e["source"]), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if h != e["sha256"]:
+        return None
+    return e["bytes_per_launch"].get(workload)
+
+
 def _peaks() -> dict:
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -66,7 +95,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except OSError:
@@ -416,7 +445,7 @@ def run_cuda(args) -> None:
     gate_gbs = gate_b / (ms_gate * 1e-3) / 1e9
 
     cpu = _oracle_layer_step_us(w, 2) if world == 1 or rank == 0 else None
-    n_split_kernels = 3  # refresh + attend + combine per skip layer-step
+    launches_per_layer_step = 1  # a skip layer-step is one launch: refresh + attention + merge
     line = {
         "metric": "us_per_layer_step_skip", "value": us_skip, "unit": "us", "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms_skip, "higher_is_better": False, "scaling": "weak",
@@ -430,19 +459,22 @@ def run_cuda(args) -> None:
                       "skip_over_recompute": us_skip / us_rec},
         "kernels_us": {"attend_skip": ms_att_skip * 1e3, "attend_recompute": ms_att_rec * 1e3,
                        "entropy_gate": ms_gate * 1e3, "kv_refresh_skip": ms_refresh * 1e3},
-        "roofline": {"kernel": "ec_attend skip path (attention + split merge)", "bound": "hbm",
+        "roofline": {"kernel": "ec_attend skip path (attend_skip_kernel: refresh + attention + merge)", "bound": "hbm",
                      "achieved": att_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": att_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+                     "frac": att_gbs / peaks["hbm_gbs"], "traffic": _ncu_traffic("attend_skip", w.name),
+                     "algorithmic_bytes": skip_b, "peak_source": peaks["source"]},
         "roofline_recompute": {"kernel": "ec_attend recompute path", "bound": "tensor", "achieved": rec_tf,
                                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                               "frac": rec_tf / peaks["bf16_tflops"], "traffic": None,
-                               "peak_source": peaks["source"]},
+                               "frac": rec_tf / peaks["bf16_tflops"],
+                               "traffic": _ncu_traffic("attend_dense", w.name), "algorithmic_flops": rec_f,
+                               "peak_source": peaks["source"] + " (burst: the kernel is timed alone)"},
         "roofline_gate": {"kernel": "ec_entropy_gate", "bound": "hbm", "achieved": gate_gbs,
                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gate_gbs / peaks["hbm_gbs"],
-                          "traffic": None, "peak_source": peaks["source"]},
+                          "traffic": _ncu_traffic("entropy_gate", w.name), "algorithmic_bytes": gate_b,
+                          "peak_source": peaks["source"]},
         "e2e": {"value": ms_e2e * 1e3 / n_layers / world, "unit": "us", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
-        "gpu_launches": K * (n_layers * n_split_kernels + 1),
+        "gpu_launches": K * (n_layers * launches_per_layer_step + 1),
         "clocks": clocks,
     }
     if cpu is not None:
