@@ -228,6 +228,17 @@ class DeviceWorkload:
         return self.R * self.w.vocab * syn.elem_bytes(self.w.dtype) + 12 * self.R
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The step time of the whole job is the slowest rank's (replicas: no other exchange between ranks)."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def _graph_time(torch, body, replays: int, warmup: int, stream) -> float:
     """Captures body() into a CUDA graph, replays it `warmup` times untimed and `replays`
     times timed; returns milliseconds per replay (CUDA events on the launching stream)."""
@@ -356,11 +367,7 @@ def run_cuda(args) -> None:
         torch.cuda.synchronize()
 
     def reduce_max(ms: float) -> float:
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks(ms, dist, dev)
 
     # ---- headline: K skip steps ----------------------------------------------------
     sampler = ClockSampler(local)

@@ -1,0 +1,112 @@
+"""GPU replays of the cached denoising loop (Algorithm 1 / Appendix A) against the fp64 oracle:
+refresh -> attend -> gate, step after step, on the same seeded tensors.  Compared per step: the
+attention output (bf16: max-abs <= 1e-2; fp32: <= 1e-5 relative), the gate's maximum entropy
+(<= 1e-4 nats) and decision (bit-exact unless |E - tau| < 1e-4, where the oracle's decision drives
+both replays); at the end: the KV caches byte for byte."""
+import numpy as np
+import pytest
+import torch
+
+import ec_synth as syn
+import oracle
+from _replay import run_replay, step_inputs, ReplayState, decoded_this_step
+from _util import to_dev, to_f64, to_storage
+
+pytestmark = pytest.mark.gpu
+
+
+def _caches(w):
+    t = syn.attn_inputs(w, w.ctx_len)
+    return t["k_cache"], t["v_cache"]
+
+
+def _oracle_fns(w, kc, vc):
+    def attend(q, kn, vn, idx):
+        return oracle.refresh_and_attend(q, kn, vn, kc, vc, idx, w.dtype)
+
+    def gate(logits, flags, tau):
+        o = oracle.entropy_gate(logits, w.dtype, w.vocab, flags, tau, w.block)
+        return o["max_entropy"][0], int(o["decision"][0])
+
+    return attend, gate
+
+
+def _gpu_fns(w, gk, gv):
+    import paper_2603_18489_b200 as ec
+
+    d = ec.make_desc(w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def attend(q, kn, vn, idx):
+        out = ec.ec_attend(d, to_dev(q), to_dev(kn), to_dev(vn), gk, gv, to_dev(idx), dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        return to_f64(out)
+
+    def gate(logits, flags, tau):
+        r = ec.ec_entropy_gate(to_dev(logits), w.vocab, w.block, to_dev(flags), tau)
+        torch.cuda.synchronize()
+        return float(r["max_entropy"][0]), int(r["decision"][0])
+
+    return attend, gate
+
+
+def _compare(w, n_steps, tau, k, sigma_centre_fn=None):
+    kc, vc = _caches(w)
+    okc, ovc = kc.copy(), vc.copy()
+    o_att, o_gate = _oracle_fns(w, okc, ovc)
+    ref = run_replay(w, n_steps, tau, k, o_att, o_gate, None, sigma_centre_fn)
+    forced = [r["decision"] for r in ref]
+    gk, gv = to_dev(kc), to_dev(vc)
+    g_att, g_gate = _gpu_fns(w, gk, gv)
+    got = run_replay(w, n_steps, tau, k, g_att, g_gate, None, sigma_centre_fn, forced_decisions=forced)
+    assert ref[0]["full"] and got[0]["full"]
+    for a, b in zip(ref, got):
+        assert a["full"] == b["full"] and a["n_active"] == b["n_active"]
+        err = np.abs(a["out"] - b["out"]).max()
+        if w.dtype == syn.BF16:
+            assert err <= 1e-2, (a["step"], err)
+        else:
+            assert err <= 1e-5 * np.abs(a["out"]).max(), (a["step"], err)
+        assert abs(a["E"] - b["E"]) <= 1e-4, (a["step"], a["E"], b["E"])
+        if abs(a["E"] - tau) >= 1e-4:
+            assert a["decision"] == b["decision"], (a["step"], a["E"], tau)
+    assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)
+    return ref
+
+
+def _tau_for_recompute_share(w, n_steps, share, sigma_centre_fn=None):
+    """tau such that about `share` of the steps exceed it: the per-step maximum entropies only depend on the
+    seeded logits and flags, so a gate-only pre-pass of the oracle gives them."""
+    st = ReplayState(w)
+    E = []
+    for s in range(n_steps):
+        centre = None if sigma_centre_fn is None else sigma_centre_fn(s)
+        lg = step_inputs(w, s, 1, centre)["logits"]
+        flags = decoded_this_step(st, s, 4)
+        if not flags.any():
+            st.masked[:] = True
+            flags = decoded_this_step(st, s, 4)
+        o = oracle.entropy_gate(lg, w.dtype, w.vocab, flags, 0.0, w.block)
+        E.append(o["max_entropy"][0])
+        st.record(flags, 0)
+    return float(np.float32(np.quantile(E, 1.0 - share)))
+
+
+def test_config1_eight_step_replay_fp32():
+    w = syn.C1
+    tau = _tau_for_recompute_share(w, 8, 0.5)          # config 1: tau = median
+    ref = _compare(w, 8, tau, w.k_recent)
+    kinds = [r["full"] for r in ref]
+    assert kinds[0] and any(kinds[1:]) and not all(kinds)      # both branches were exercised
+
+
+@pytest.mark.parametrize("k", [2, 8])
+def test_config4_block_replay_with_drifting_sigma(k):
+    w = syn.C4
+    centre = lambda s: syn.drifting_sigma_centre(s)
+    tau = _tau_for_recompute_share(w, 32, 0.15, centre)
+    ref = _compare(w, 32, tau, k, centre)
+    n_full = sum(r["full"] for r in ref)
+    assert 2 <= n_full <= 12
+    assert all(r["n_active"] in (w.ctx_len,) or 32 <= r["n_active"] <= 32 + 32 for r in ref)
