@@ -343,6 +343,9 @@ def run_cuda(args) -> None:
     w = syn.WORKLOADS[args.workload]
     n_layers = args.layers or _choose_layers(w)
     peaks = _peaks()
+    if args.trace:
+        _run_trace(args, torch, w, dev)
+        return
     if args.only:
         _run_only(args, torch, w, n_layers, dev)
         return
@@ -495,6 +498,120 @@ def run_cuda(args) -> None:
         dist.destroy_process_group()
 
 
+def _run_trace(args, torch, w, dev) -> None:
+    """Full-depth step trace (the fifth benchmark configuration): n_layers layers, every sequence of the batch
+    with its own skip / recompute decision taken by ec_entropy_gate on that step's logits, the host reading
+    the decisions back every step as the generation loop does (Algorithm 1).  Logits are seeded Gaussian rows
+    whose sigma band drifts from step to step (a different phase per sequence); tau is set from a gate-only
+    pre-pass so that about 15 % of the sequence-steps recompute (the paper's recompute ratios are 0.11-0.18).
+    Prints one JSON line: time per step by kind and the skip / recompute cost per layer-step and sequence."""
+    import paper_2603_18489_b200 as ec
+
+    B, L, Hq, Hkv, D, V = w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.vocab
+    n_layers = args.layers or w.n_layers
+    n_steps = w.n_steps if w.n_steps > 1 else 16
+    dt = torch.bfloat16 if w.dtype == syn.BF16 else torch.float32
+    g = torch.Generator(device=dev)
+    g.manual_seed(4321)
+    std = 1.0 / np.sqrt(D)
+
+    def rn(*shape):
+        return (torch.randn(*shape, generator=g, device=dev, dtype=torch.float32) * std).to(dt)
+
+    kc = [rn(B, Hkv, L, D) for _ in range(n_layers)]
+    vc = [rn(B, Hkv, L, D) for _ in range(n_layers)]
+    n = w.n_skip_rows
+    q_s, kn_s, vn_s = rn(B, n, Hq, D), rn(B, n, Hkv, D), rn(B, n, Hkv, D)
+    q_r, kn_r, vn_r = rn(B, L, Hq, D), rn(B, L, Hkv, D), rn(B, L, Hkv, D)
+    out_s, out_r = torch.empty_like(q_s), torch.empty_like(q_r)
+    idx = torch.from_numpy(syn.active_rows(w, block_no=(w.gen_len // w.block) // 2)).to(dev)
+    d1 = ec.make_desc(1, L, Hq, Hkv, D, w.dtype)
+    dB = ec.make_desc(B, L, Hq, Hkv, D, w.dtype)
+    ws = ec.new_workspace(max(ec.ec_attend_workspace_bytes(dB, n), ec.ec_attend_workspace_bytes(dB, L)), dev)
+    R = B * w.block
+    period = 16
+    logits = []
+    for s_ in range(period):
+        rows = []
+        for b in range(B):
+            centre = syn.drifting_sigma_centre(s_ + 2 * b, period)
+            sig = torch.rand(w.block, 1, generator=g, device=dev) * 3.0 + max(0.25, centre - 1.5)
+            rows.append((torch.randn(w.block, V, generator=g, device=dev) * sig).to(dt))
+        logits.append(torch.cat(rows, 0))
+    flags = torch.from_numpy(syn.decoded_flags(R, 4, w.block, cfg_id=w.cfg_id)).to(dev)
+    ws_g = ec.new_workspace(ec.ec_entropy_gate_workspace_bytes(R, V), dev)
+    maxh = torch.empty(B, device=dev, dtype=torch.float32)
+    dec = torch.empty(B, device=dev, dtype=torch.int32)
+    # tau from a gate-only pre-pass: the 85th percentile of the per-(step, sequence) maximum entropies
+    E = []
+    for lg in logits:
+        ec.ec_entropy_gate(lg, V, w.block, flags, 0.0, max_entropy_out=maxh, decision_out=dec, workspace=ws_g,
+                           want_rows=False)
+        E.append(maxh.cpu().numpy().copy())
+    tau = float(np.quantile(np.concatenate(E), 0.85))
+
+    def attend(group, full: bool, layer: int):
+        """One ec_attend per maximal run of consecutive sequences of the group."""
+        calls = 0
+        i = 0
+        while i < len(group):
+            j = i
+            while j + 1 < len(group) and group[j + 1] == group[j] + 1:
+                j += 1
+            b0, nb = group[i], j - i + 1
+            d = ec.make_desc(nb, L, Hq, Hkv, D, w.dtype)
+            sl = slice(b0, b0 + nb)
+            if full:
+                ec.ec_attend(d, q_r[sl], kn_r[sl], vn_r[sl], kc[layer][sl], vc[layer][sl], None, out=out_r[sl],
+                             workspace=ws)
+            else:
+                ec.ec_attend(d, q_s[sl], kn_s[sl], vn_s[sl], kc[layer][sl], vc[layer][sl], idx[sl], out=out_s[sl],
+                             workspace=ws)
+            calls += 1
+            i = j + 1
+        return calls
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    decisions = np.ones(B, np.int64)   # step 1 is a full pass for every sequence
+    t_skip = t_rec = t_gate = 0.0
+    n_skip = n_rec = launches = 0
+    per_step = []
+    torch.cuda.synchronize()
+    for s_ in range(n_steps):
+        sk = [b for b in range(B) if decisions[b] == 0]
+        rc = [b for b in range(B) if decisions[b] != 0]
+        e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+        e0.record()
+        for l in range(n_layers):
+            launches += attend(sk, False, l)
+        e1.record()
+        for l in range(n_layers):
+            launches += 2 * attend(rc, True, l)
+        e2.record()
+        ec.ec_entropy_gate(logits[s_ % period], V, w.block, flags, tau, max_entropy_out=maxh, decision_out=dec,
+                           workspace=ws_g, want_rows=False)
+        e3.record()
+        decisions = dec.cpu().numpy().astype(np.int64)   # the host reads the decisions: they shape the next step
+        launches += 1
+        a, b_, c = e0.elapsed_time(e1) * 1e3, e1.elapsed_time(e2) * 1e3, e2.elapsed_time(e3) * 1e3
+        if s_ > 0:   # the all-recompute first step warms everything up and is reported apart
+            t_skip += a; t_rec += b_; t_gate += c
+            n_skip += len(sk); n_rec += len(rc)
+        per_step.append(dict(step=s_, n_skip=len(sk), n_recompute=len(rc), us=a + b_ + c))
+    us_skip = t_skip / max(n_skip * n_layers, 1)
+    us_rec = t_rec / max(n_rec * n_layers, 1)
+    print(json.dumps({
+        "trace": w.name, "n_layers": n_layers, "n_steps": n_steps, "batch": B, "tau": tau,
+        "recompute_fraction": n_rec / max(n_skip + n_rec, 1),
+        "us_per_layer_step_sequence": {"skip": us_skip, "recompute": us_rec},
+        "skip_over_recompute": us_skip / us_rec if us_rec > 0 else None,
+        "us_per_step_mean": {"attend_skip": t_skip / max(n_steps - 1, 1), "attend_recompute": t_rec / max(n_steps - 1, 1),
+                             "gate": t_gate / max(n_steps - 1, 1)},
+        "first_step_us": per_step[0]["us"], "gpu_launches": launches,
+        "pattern": "".join("R" if p_["n_recompute"] == B else ("s" if p_["n_recompute"] == 0 else "m") for p_ in per_step),
+        "timing": "CUDA events per step on the current stream, plain launches, host reads the decisions every step"}))
+
+
 def _run_only(args, torch, w, n_layers: int, dev) -> None:
     """Profiling aid: one part of the step over the same device workload (one CUDA graph
     per step, like the full run), a few iterations, one short JSON line."""
@@ -517,6 +634,8 @@ def main() -> None:
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(syn.WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="distinct K/V caches per step (0: enough to exceed 3x L2)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--trace", action="store_true",
+                    help="full-depth step trace of the workload (its layers and steps; decisions from the gate)")
     ap.add_argument("--only", default="", choices=["", "skip", "recompute", "gate"],
                     help="profiling aid: run only this part of the step")
     args = ap.parse_args()
