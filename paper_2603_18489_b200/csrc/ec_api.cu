@@ -26,19 +26,24 @@ namespace {
 
 // bf16 with head_dim 128 runs on the tcgen05 kernels (the fused skip-step kernel when the packed
 // query rows fit two M tiles, the dense kernel otherwise); everything else bf16 on the mma.sync kernel.
-// EC_ATTEND_IMPL (environment, read once) = "mma" forces the mma.sync kernel, "dense" the dense
-// tcgen05 kernel with a separate refresh launch: for A/B measurements only.
+// EC_ATTEND_IMPL (environment, read once) = "mma" forces the mma.sync kernel, "dense" the one-tile dense
+// tcgen05 kernel with a separate refresh launch, "rows" the skip kernel with query rows on the M axis: for A/B
+// measurements only.
 int forced_impl() {
     static const int f = [] {
         const char* e = std::getenv("EC_ATTEND_IMPL");
         if (e && std::strcmp(e, "mma") == 0) return 1;
         if (e && std::strcmp(e, "dense") == 0) return 2;
+        if (e && std::strcmp(e, "rows") == 0) return 3;
         return 0;
     }();
     return f;
 }
 bool use_tc(const ec_attn_desc& d) { return d.dtype == EC_BF16 && d.head_dim == 128 && forced_impl() != 1; }
-bool use_skip(const ec_attn_desc& d, int n_active) { return forced_impl() == 0 && attend_skip_supported(d, n_active); }
+bool use_skip_keys(const ec_attn_desc& d, int n_active) { return forced_impl() == 0 && attend_skip_keys_supported(d, n_active); }
+bool use_skip(const ec_attn_desc& d, int n_active) {
+    return (forced_impl() == 0 || forced_impl() == 3) && attend_skip_supported(d, n_active);
+}
 
 size_t attend_ws(const ec_attn_desc& d, int n_active) {
     size_t n = attend_workspace_bytes(d, n_active);
@@ -113,7 +118,8 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
     if (!aligned16(workspace)) return EC_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool fused = use_skip(*desc, n_active);
+    const bool fused_keys = use_skip_keys(*desc, n_active);
+    const bool fused = fused_keys || use_skip(*desc, n_active);
 
     if (k_new && !fused) {
         if (launch_refresh(*desc, k_cache, v_cache, k_new, v_new, active_idx, n_active, s) != cudaSuccess)
@@ -130,7 +136,8 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     a.workspace_bytes = workspace_bytes;
     a.dev_status = dev_status;
     a.scale = desc->scale > 0.f ? desc->scale : 1.0f / sqrtf((float)desc->head_dim);
-    const cudaError_t e = fused                  ? launch_attend_skip(a, k_new, v_new, active_idx, s)
+    const cudaError_t e = fused_keys             ? launch_attend_skip_keys(a, k_new, v_new, active_idx, s)
+                          : fused                ? launch_attend_skip(a, k_new, v_new, active_idx, s)
                           : desc->dtype != EC_BF16 ? launch_attend_f32(a, s)
                           : (use_tc(*desc) && forced_impl() != 2 && attend_dense_supported(*desc, n_active)) ? launch_attend_dense(a, s)
                           : use_tc(*desc)        ? launch_attend_bf16_tc(a, s)

@@ -73,6 +73,10 @@ cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);      /
 bool attend_skip_supported(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                cudaStream_t stream);
+// skip-step path with the keys on the M axis (bf16, head_dim 128, n_active * H_q/H_kv <= 64)
+bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active);
+cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
+                                    cudaStream_t stream);
 // two-row-tile dense path (bf16, head_dim 128): used when its (row-tile pair, kv head) units fill the GPU
 bool attend_dense_supported(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream);
