@@ -44,9 +44,9 @@ DEFAULT_WORKLOAD = "c2_llada_l768"
 # profiles/.  A figure is reported only while the kernel's source file still has the hash it had when the
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
-    "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
-                    "sha256": "33bdbd0bbaf1065a8524d965ba870f214f2555de4dc95aa6cd23f979c5b9fcdb",
-                    "bytes_per_launch": {"c2_llada_l768": 12930816, "c5_llada_l4096": 68199168}},
+    "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
+                    "sha256": "capture pending",
+                    "bytes_per_launch": {}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
                      "sha256": "8b9b93fb78eb526dd48d92e6b73050e6a46dcac25c98baaf4c4c32f7162da1d1",
                      "bytes_per_launch": {"c4_llada_l2048": 51188992, "c5_llada_l4096": 116217856}},
@@ -469,7 +469,7 @@ def run_cuda(args) -> None:
                       "skip_over_recompute": us_skip / us_rec},
         "kernels_us": {"attend_skip": ms_att_skip * 1e3, "attend_recompute": ms_att_rec * 1e3,
                        "entropy_gate": ms_gate * 1e3, "kv_refresh_skip": ms_refresh * 1e3},
-        "roofline": {"kernel": "ec_attend skip path (attend_skip_kernel: refresh + attention + merge)", "bound": "hbm",
+        "roofline": {"kernel": "ec_attend skip path (one launch: refresh + attention + merge)", "bound": "hbm",
                      "achieved": att_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": att_gbs / peaks["hbm_gbs"], "traffic": _ncu_traffic("attend_skip", w.name),
                      "algorithmic_bytes": skip_b, "peak_source": peaks["source"]},

@@ -47,8 +47,8 @@ constexpr int kMaxRowsT = 64;
 constexpr uint32_t TM_COLS = 256;          // S^T buffers at columns 0 and 64, O^T at 128
 constexpr uint32_t TM_S = 0, TM_O = 128;
 // exchange areas, reusing the dead staging memory after the main loop (bytes from the aligned base)
-constexpr uint32_t kStagingOff = 32768;                       // row-sum scratch [128][N] floats sits below it
-constexpr uint32_t kExchangeMax = (128 * 64 + 2 * 64 * 8) * 4;   // C chunks of (128/C) x N + 2N floats, N <= 64, C <= 8
+constexpr uint32_t kStagingOff = 36864;                       // row-sum scratch [128][N + 1] floats sits below it
+constexpr uint32_t kExchangeMax = (128 * 65 + 2 * 64 * 8) * 4;   // C chunks of (128/C) x (N + 1) + 2N floats, N <= 64, C <= 8
 constexpr uint32_t kRecvOff = kStagingOff + 40960;
 
 enum { B_FULL = 0, B_EMPTY = kMaxStages, B_SFULL = 2 * kMaxStages, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 1,
@@ -99,6 +99,7 @@ struct KeysParams {
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
     int n_splits, tiles_per_split, n_stages;
+    int q_tma;                    // 1: the producer fetches Q with one TMA box (MHA); 0: the softmax warps stage it
     uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0
     float scale_log2;
 };
@@ -117,7 +118,8 @@ struct alignas(16) KeysShared {
 
 template <int N>
 __global__ void __launch_bounds__(kThreads, 1)
-attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const KeysParams p) {
+attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                        const __grid_constant__ CUtensorMap map_q, const KeysParams p) {
     static_assert(N == 48 || N == 64, "query-row slots per CTA");
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (s2u(smem_raw) + 1023u) & ~1023u;
@@ -139,15 +141,17 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int T = t_end - t_begin;   // >= 1 by construction of the plan
     const int NS = p.n_stages;
     const bool refresh = p.k_new != nullptr;
-    const uint32_t chunk_bytes = (uint32_t)(DL * N + 2 * N) * 4u;   // one owner's slice of O^T, then m[N], l[N]
+    constexpr int NP = N + 1;   // odd row stride (floats) of the transposing buffers: conflict-free by row and by column
+    const uint32_t chunk_bytes = (uint32_t)(DL * NP + 2 * N) * 4u;   // one owner's slice of O^T, then m[N], l[N]
 
     // ---- set-up (touches no global memory) -------------------------------------------------
     if (tid == 0) {
         prefetch_map(&map_k);
         prefetch_map(&map_v);
+        if (p.q_tma) prefetch_map(&map_q);
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1;
-            if (i == B_PFULL || i == B_QFULL || i == B_REFRESHED) count = kSoft;
+            if (i == B_PFULL || i == B_REFRESHED || (i == B_QFULL && !p.q_tma)) count = kSoft;
             mbar_init(bar(i), count);
         }
         sh->abort_flag = 0;
@@ -175,6 +179,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     if (warp == 0) {
         // ================================ TMA producer ======================================
         if (lane == 0) {
+            if (p.q_tma) {   // Q first: [half][row][64 columns] of this head's rows, rows past n_active read as zero
+                mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
+                tma_load_5d(base, &map_q, 0, 0, hk, 0, b, bar(B_QFULL));
+            }
             int first_tile = 0, j_refreshed = T;
             if (refresh) {
                 mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
@@ -275,7 +283,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         const int stid = tid - 64;
         constexpr uint32_t QHALF = N * 128;
         // Q rows of this kv head -> swizzled K-major tile of N rows (rows past rows_total are zero)
-        for (int c = stid; c < N * (HD / 8); c += kSoft) {
+        for (int c = stid; c < (p.q_tma ? 0 : N * (HD / 8)); c += kSoft) {
             const int row = c >> 4, ch = c & 15;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             if (row < p.rows_total) {
@@ -286,8 +294,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             const uint32_t off = (ch >> 3) * QHALF + (row >> 3) * 1024 + (row & 7) * 128 + (((ch & 7) ^ (row & 7)) << 4);
             *reinterpret_cast<uint4*>(gbase + off) = v;
         }
-        fence_async_smem();         // Q (generic proxy) -> visible to the tensor core (async proxy)
-        mbar_arrive(bar(B_QFULL));
+        if (!p.q_tma) {
+            fence_async_smem();     // Q (generic proxy) -> visible to the tensor core (async proxy)
+            mbar_arrive(bar(B_QFULL));
+        }
 
         int first_tile = 0;
         if (refresh) {
@@ -423,19 +433,27 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         fence_after();
 
         // ---- row sums over the CTA's keys: per-thread partials -> shared memory -> one thread per query ----
-        float* lred = reinterpret_cast<float*>(gbase);   // [128 keys][N]
+        float* lred = reinterpret_cast<float*>(gbase);   // [128 keys][NP]
 #pragma unroll
         for (int i = 0; i < N / 2; ++i) {
             float a0, a1;
             upk(l2[i], a0, a1);
-            *reinterpret_cast<float2*>(lred + kk * N + 2 * i) = make_float2(a0, a1);
+            lred[kk * NP + 2 * i] = a0;
+            lred[kk * NP + 2 * i + 1] = a1;
         }
         named_barrier(3, kSoft);
-        if (stid < N) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-            for (int k = 0; k < BK; ++k) acc[k & 3] += lred[k * N + stid];
-            sh->factor[stid] = (acc[0] + acc[1]) + (acc[2] + acc[3]);   // l[q] of this CTA
+        {   // two threads per query column, 64 keys each
+            const int qc = stid & 63, half = stid >> 6;
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (qc < N) {
+#pragma unroll
+                for (int k = 0; k < 64; ++k) acc[k & 7] += lred[(half * 64 + k) * NP + qc];
+            }
+            const float part = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+            named_barrier(3, kSoft);   // every partial sum has been read out of lred
+            if (qc < N) lred[half * N + qc] = part;
+            named_barrier(3, kSoft);
+            if (stid < N) sh->factor[stid] = lred[stid] + lred[N + stid];   // l[q] of this CTA
         }
         named_barrier(3, kSoft);
 
@@ -458,14 +476,12 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             }
         } else {
             // ---- this CTA's O^T row kk -> staging chunk of the CTA that owns output column kk ----
-            float* stg = reinterpret_cast<float*>(gbase + kStagingOff) + (kk / DL) * (chunk_bytes / 4) + (kk % DL) * N;
+            float* stg = reinterpret_cast<float*>(gbase + kStagingOff) + (kk / DL) * (chunk_bytes / 4) + (kk % DL) * NP;
 #pragma unroll
-            for (int c = 0; c < N; c += 4)
-                *reinterpret_cast<float4*>(stg + c) = make_float4(__uint_as_float(o[c]), __uint_as_float(o[c + 1]),
-                                                                  __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
+            for (int c = 0; c < N; ++c) stg[c] = __uint_as_float(o[c]);
             if (stid < N) {   // every owner also gets this CTA's m[q] and l[q]
                 for (int c = 0; c < C; ++c) {
-                    float* ml = reinterpret_cast<float*>(gbase + kStagingOff) + c * (chunk_bytes / 4) + DL * N;
+                    float* ml = reinterpret_cast<float*>(gbase + kStagingOff) + c * (chunk_bytes / 4) + DL * NP;
                     ml[stid] = sh->m[stid];
                     ml[N + stid] = sh->factor[stid];
                 }
@@ -490,19 +506,30 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         mbar_wait(bar(B_RECV), 0, abort_flag, p.dev_status);
         const float* recv = reinterpret_cast<const float*>(gbase + kRecvOff);
         const int cf = (int)(chunk_bytes / 4);
-        const int dl = tid % DL;
-        for (int qq = tid / DL; qq < p.rows_total; qq += kThreads / DL) {
+        float* wgt = reinterpret_cast<float*>(gbase);   // [C][N] normalised weights 2^(m_s - m) / l, over the dead row-sum scratch
+        long long* qoff = reinterpret_cast<long long*>(gbase + 4096);   // [N] element offset of each query row in out
+        if (tid < N) {
             float m = -INFINITY;
-            for (int s = 0; s < C; ++s) m = fmaxf(m, recv[s * cf + DL * N + qq]);
-            float acc = 0.f, l = 0.f;
+            for (int s = 0; s < C; ++s) m = fmaxf(m, recv[s * cf + DL * NP + tid]);
+            float l = 0.f;
+            for (int s = 0; s < C; ++s) l = fmaf(fast_exp2(recv[s * cf + DL * NP + tid] - m), recv[s * cf + DL * NP + N + tid], l);
+            const float inv = 1.f / l;
+            for (int s = 0; s < C; ++s) wgt[s * N + tid] = fast_exp2(recv[s * cf + DL * NP + tid] - m) * inv;
+            const int i = tid / p.group, jh = tid % p.group;
+            qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + split * DL;
+        }
+        __syncthreads();
+        // a thread owns two adjacent output columns of a query row: one 4-byte store
+        const int half_dl = DL / 2;
+        const int dp = tid % half_dl;
+        for (int qq = tid / half_dl; qq < p.rows_total; qq += kThreads / half_dl) {
+            float a0 = 0.f, a1 = 0.f;
             for (int s = 0; s < C; ++s) {
-                const float w = fast_exp2(recv[s * cf + DL * N + qq] - m);
-                l = fmaf(w, recv[s * cf + DL * N + N + qq], l);
-                acc = fmaf(w, recv[s * cf + dl * N + qq], acc);
+                const float w = wgt[s * N + qq];
+                a0 = fmaf(w, recv[s * cf + (2 * dp) * NP + qq], a0);
+                a1 = fmaf(w, recv[s * cf + (2 * dp + 1) * NP + qq], a1);
             }
-            const int i = qq / p.group, jh = qq % p.group;
-            p.out[(((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + split * DL + dl] =
-                __float2bfloat16_rn(acc / l);
+            *reinterpret_cast<uint32_t*>(p.out + qoff[qq] + 2 * dp) = pack_bf16x2(a0, a1);
         }
         // no CTA leaves while a peer may still copy out of or into its shared memory
         __syncwarp();
@@ -550,6 +577,21 @@ bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// q [B, n, H_q, 128] bf16 (MHA: one query head per kv head) seen as 5-D {64 columns, row, head, half, sequence}:
+// the box {64, N, 1, 2, 1} lands as [half][row][64 columns], the K-major Q tile; rows past n read as zero
+bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_q_heads, int n_slots) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[5] = {64, (cuuint64_t)n_active, (cuuint64_t)n_q_heads, 2, (cuuint64_t)batch};
+    const cuuint64_t strides[4] = {(cuuint64_t)n_q_heads * HD * 2, (cuuint64_t)HD * 2, 128,
+                                   (cuuint64_t)n_active * n_q_heads * HD * 2};
+    const cuuint32_t box[5] = {64, (cuuint32_t)n_slots, 1, 2, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct KeysPlan {
     int n_slots, n_splits, tiles_per_split, n_stages;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
@@ -592,8 +634,8 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
 }
 
 template <int N>
-cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv, int bh,
-                     cudaStream_t stream) {
+cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv,
+                     const CUtensorMap& mq, int bh, cudaStream_t stream) {
     static bool attr_done[64] = {};   // the attribute is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
@@ -617,7 +659,7 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, p);
+    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, mq, p);
 }
 
 }  // namespace
@@ -629,6 +671,8 @@ bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
     if ((long long)d.batch * d.n_kv_heads > 65535) return false;   // grid.y
     const KeysPlan pl = make_keys_plan(d, n_active);
     // the exchange areas (row-sum scratch, staging, receive buffer) reuse the memory below the refresh list
+    // one CTA per SM: beyond one wave of CTAs the row-major skip kernel (two CTAs per SM) streams better
+    if ((long long)pl.n_splits * d.batch * d.n_kv_heads > sm_count()) return false;
     return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && kRecvOff + kExchangeMax <= pl.off_list;
 }
 
@@ -640,6 +684,9 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
         return cudaErrorInvalidValue;
     KeysParams p{};
+    CUtensorMap map_q = map_k;   // unused unless q_tma
+    p.q_tma = (a.d.n_q_heads == a.d.n_kv_heads) ? 1 : 0;
+    if (p.q_tma && !make_q_map(&map_q, a.q, a.d.batch, a.n_active, a.d.n_q_heads, pl.n_slots)) return cudaErrorInvalidValue;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
     p.v_new = static_cast<const __nv_bfloat16*>(v_new);
@@ -662,7 +709,8 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.off_list = pl.off_list;
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
-    return pl.n_slots == 48 ? launch_n<48>(pl, p, map_k, map_v, bh, stream) : launch_n<64>(pl, p, map_k, map_v, bh, stream);
+    return pl.n_slots == 48 ? launch_n<48>(pl, p, map_k, map_v, map_q, bh, stream)
+                            : launch_n<64>(pl, p, map_k, map_v, map_q, bh, stream);
 }
 
 }  // namespace ec
