@@ -136,3 +136,29 @@ def test_key_permutation_invariance_on_device():
     t2["v_cache"] = np.ascontiguousarray(t["v_cache"][:, :, perm])
     out1, _, _ = _gpu_attend(w, t2, refresh=False)
     assert np.abs(to_f64(out0) - to_f64(out1)).max() <= 2e-3
+
+
+@pytest.mark.parametrize("Hq,Hkv,n,L", [(8, 8, 56, 1000), (8, 8, 64, 512), (8, 4, 30, 700), (6, 2, 21, 259),
+                                        (32, 32, 48, 2048), (4, 4, 49, 129), (16, 16, 34, 4096)])
+def test_few_row_skip_steps_through_both_slot_counts(Hq, Hkv, n, L):
+    """Skip steps whose packed query rows (n x H_q/H_kv <= 64) take the kernel with the keys on the M axis:
+    48 and 64 query slots, MHA (Q by TMA) and GQA (Q staged by threads), ragged last key tile, one to eight
+    CTAs per head, refreshed rows scattered over the context."""
+    w = syn.Workload(94, "fewrows", syn.BF16, 2, Hq, Hkv, 128, 0, L, 1, 0, 64)
+    idx = syn.arbitrary_active_idx(2, L, n, seed=7 * L + n)
+    t = syn.attn_inputs(w, n, active_idx=idx, std_qk=0.7, std_v=0.5)
+    _check(w, t)
+    _check(w, t, refresh=False)
+
+
+def test_few_row_skip_step_with_rising_maxima():
+    """Keys ordered so that the row maxima keep rising from tile to tile (scores grow with the position): the
+    lazily updated references must be raised, and the accumulator rescaled, several times."""
+    w = syn.Workload(93, "rising", syn.BF16, 1, 4, 4, 128, 0, 1024, 1, 0, 64)
+    t = syn.attn_inputs(w, 40, active_idx=syn.arbitrary_active_idx(1, 1024, 40, seed=3), std_qk=0.3, std_v=0.5)
+    q = syn.decode_f64(t["q"], syn.BF16)
+    k = syn.decode_f64(t["k_cache"], syn.BF16)
+    ramp = np.linspace(0.0, 3.0, 1024)[None, None, :, None]            # key j carries j/341 of the mean query direction
+    k = k + ramp * q.mean(axis=1)[:, :, None, :] * 8.0
+    t["k_cache"] = syn.encode(k.astype(np.float32), syn.BF16)
+    _check(w, t, scale=1.0, refresh=False)
