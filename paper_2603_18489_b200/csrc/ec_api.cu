@@ -121,7 +121,11 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     const bool fused_keys = use_skip_keys(*desc, n_active);
     const bool fused = fused_keys || use_skip(*desc, n_active);
 
-    if (k_new && !fused) {
+    const bool dense = !fused && use_tc(*desc) && forced_impl() != 2 && attend_dense_supported(*desc, n_active);
+    // recompute step on the dense path: every cache row is overwritten by the fresh row of the same position, so
+    // attention reads K/V straight from k_new / v_new and a spare warp of the same launch copies them into the cache
+    const bool from_new = dense && k_new && !active_idx;
+    if (k_new && !fused && !from_new) {
         if (launch_refresh(*desc, k_cache, v_cache, k_new, v_new, active_idx, n_active, s) != cudaSuccess)
             return EC_ERR_CUDA;
     }
@@ -136,10 +140,17 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     a.workspace_bytes = workspace_bytes;
     a.dev_status = dev_status;
     a.scale = desc->scale > 0.f ? desc->scale : 1.0f / sqrtf((float)desc->head_dim);
+    if (from_new) {
+        a.k_cache = k_new;
+        a.v_cache = v_new;
+        a.kv_token_major = true;
+        a.refresh_k_dst = k_cache;
+        a.refresh_v_dst = v_cache;
+    }
     const cudaError_t e = fused_keys             ? launch_attend_skip_keys(a, k_new, v_new, active_idx, s)
                           : fused                ? launch_attend_skip(a, k_new, v_new, active_idx, s)
                           : desc->dtype != EC_BF16 ? launch_attend_f32(a, s)
-                          : (use_tc(*desc) && forced_impl() != 2 && attend_dense_supported(*desc, n_active)) ? launch_attend_dense(a, s)
+                          : dense                ? launch_attend_dense(a, s)
                           : use_tc(*desc)        ? launch_attend_bf16_tc(a, s)
                                                  : launch_attend_bf16(a, s);
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;

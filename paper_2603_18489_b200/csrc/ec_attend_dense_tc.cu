@@ -20,6 +20,9 @@
 //               rescaled when a row maximum grows by more than 2^8 (the stale maximum stays the reference
 //               otherwise).  Halving the per-thread row shortens the softmax that sits between two uses of
 //               the tensor pipe for the same row tile.
+//   warp 18     recompute steps only: every cache row is overwritten by the fresh row of the same position, so the
+//               launch reads K/V straight from the token-major k_new / v_new (only the tensor map's strides
+//               differ) and this warp copies them into the cache meanwhile: no separate refresh pass.
 // TMEM (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,384), O_1 [384,512).
 // Shared memory: Q_0, Q_1 (32 KB each, staged once), five 32 KB K/V slots, barriers: 225 KB, one CTA per SM.
 // Every mbarrier wait is bounded; a wait that runs out sets EC_ERR_TIMEOUT in the caller's dev_status word and
@@ -34,7 +37,7 @@ using namespace tc;
 
 constexpr int BM = 128, BN = 128, HD = 128;
 constexpr int kSoftThreads = 512;          // four softmax warpgroups: (row tile) x (64-column half)
-constexpr int kThreads = 64 + kSoftThreads;
+constexpr int kThreads = 64 + kSoftThreads + 32;   // + one warp that copies fresh K/V into the cache (recompute steps)
 constexpr int kPolyOf5 = 0;                // pairs out of every five whose exponentials go to the FMA pipe
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
@@ -102,6 +105,12 @@ __device__ __forceinline__ void exp2_poly2(f32x2 d2, float& e0, float& e1) {
 struct DenseParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
+    // recompute step: the K/V this launch reads are the token-major fresh tensors [B, L, Hkv, 128]; its copy warp
+    // writes them into the caches [B, Hkv, L, 128] (nullptr: nothing to copy)
+    const uint4* k_src;
+    const uint4* v_src;
+    uint4* k_dst;
+    uint4* v_dst;
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
     float scale_log2;
@@ -156,7 +165,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const int slot = n % kSlots, u = n / kSlots;
                 if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
                 mbar_expect_tx(bar(B_FULL + slot), TILE);
-                tma_load_4d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, bh, bar(B_FULL + slot));
+                tma_load_5d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, hk, b, bar(B_FULL + slot));
             }
         }
     } else if (warp == 1) {
@@ -197,7 +206,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 if (j + 1 < T) commit(bar(B_EMPTY + (2 * j + 2) % kSlots));   // K_{j+1}
             }
         }
-    } else {
+    } else if (warp < 2 + kSoftThreads / 32) {
         // ====================== Q staging, then softmax (warps 2..17) ========================
         const int stid = tid - 64;
         // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
@@ -336,6 +345,36 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
         }
         fence_before();
+    } else if (p.k_dst != nullptr) {
+        // ====================== copy warp: this CTA's share of the refresh ============================
+        // The (row-tile pair, kv head) CTAs of a head split its positions evenly; a position's K and V rows
+        // (256 bytes each) go from [b, pos, hk, :] to [b, hk, pos, :].  Two rows per warp instruction, eight
+        // instructions in flight.  Nobody reads the cache in this launch.
+        const int n_pairs = gridDim.x;
+        const int per = (p.ctx_len + n_pairs - 1) / n_pairs;
+        const int pos0 = pair * per, pos1 = min(p.ctx_len, pos0 + per);
+        const int sub = lane >> 4, piece = lane & 15;
+        for (int pos = pos0; pos < pos1; pos += 16) {
+            uint4 kv[8], vv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int pp = pos + 2 * u + sub;
+                if (pp < pos1) {
+                    const long long src = (((long long)b * p.ctx_len + pp) * p.n_kv_heads + hk) * 16 + piece;
+                    kv[u] = __ldg(p.k_src + src);
+                    vv[u] = __ldg(p.v_src + src);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int pp = pos + 2 * u + sub;
+                if (pp < pos1) {
+                    const long long dst = (((long long)b * p.n_kv_heads + hk) * p.ctx_len + pp) * 16 + piece;
+                    p.k_dst[dst] = kv[u];
+                    p.v_dst[dst] = vv[u];
+                }
+            }
+        }
     }
 
     __syncthreads();
@@ -363,16 +402,20 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// cache [B*Hkv, L, 128] bf16 seen as 4-D {64 columns, key, half, head}: one box {64, 128, 2, 1} lands as
-// [half][key][64 columns], the two 128-byte-swizzled halves of a [128 keys x 128] tile; keys beyond L read as zero
-bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
+// K or V seen as 5-D {64 columns, key, half, kv head, sequence}: one box {64, 128, 2, 1, 1} lands as
+// [half][key][64 columns], the two 128-byte-swizzled halves of a [128 keys x 128] tile; keys beyond L read as zero.
+// Cache layout [B, Hkv, L, 128] or token-major [B, L, Hkv, 128] (the fresh K/V of a recompute step): only the
+// strides differ.
+bool make_kv_map(CUtensorMap* map, const void* ptr, int batch, int n_kv_heads, int ctx_len, bool token_major) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[4] = {64, (cuuint64_t)ctx_len, 2, (cuuint64_t)bh};
-    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)ctx_len * HD * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)BN, 2, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(cache), dims, strides, box, estr,
+    const cuuint64_t row = (cuuint64_t)HD * 2;
+    const cuuint64_t dims[5] = {64, (cuuint64_t)ctx_len, 2, (cuuint64_t)n_kv_heads, (cuuint64_t)batch};
+    const cuuint64_t strides[4] = {token_major ? row * n_kv_heads : row, 128, token_major ? row : row * ctx_len,
+                                   row * ctx_len * n_kv_heads};
+    const cuuint32_t box[5] = {64, (cuuint32_t)BN, 2, 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -392,11 +435,17 @@ bool attend_dense_supported(const ec_attn_desc& d, int n_active) {
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     const int bh = a.d.batch * a.d.n_kv_heads;
     CUtensorMap map_k, map_v;
-    if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
+    if (!make_kv_map(&map_k, a.k_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major) ||
+        !make_kv_map(&map_v, a.v_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major))
         return cudaErrorInvalidValue;
     DenseParams p;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     p.out = static_cast<__nv_bfloat16*>(a.out);
+    const bool copy = a.kv_token_major && a.refresh_k_dst && a.refresh_v_dst;
+    p.k_src = copy ? static_cast<const uint4*>(a.k_cache) : nullptr;
+    p.v_src = copy ? static_cast<const uint4*>(a.v_cache) : nullptr;
+    p.k_dst = copy ? static_cast<uint4*>(a.refresh_k_dst) : nullptr;
+    p.v_dst = copy ? static_cast<uint4*>(a.refresh_v_dst) : nullptr;
     p.dev_status = a.dev_status;
     p.n_active = a.n_active;
     p.ctx_len = a.d.ctx_len;

@@ -65,6 +65,12 @@ struct AttendArgs {
     size_t workspace_bytes;
     int32_t* dev_status;
     float scale;  // resolved (never 0)
+    // dense path only: k_cache / v_cache point at token-major tensors [batch, ctx_len, n_kv_heads, head_dim]
+    // (the fresh K/V of a recompute step) instead of the cache layout
+    bool kv_token_major = false;
+    // with kv_token_major: the caches those tensors are copied into by the same launch (nullptr: no copy)
+    void* refresh_k_dst = nullptr;
+    void* refresh_v_dst = nullptr;
 };
 size_t attend_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_f32(const AttendArgs& a, cudaStream_t stream);
