@@ -45,11 +45,11 @@ DEFAULT_WORKLOAD = "c2_llada_l768"
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
     "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-                    "sha256": "capture pending",
-                    "bytes_per_launch": {}},
+                    "sha256": "bb56071265acf609b4de4ef099da6642e6a7bdacb777b76370e8e1f4dca5bb13",
+                    "bytes_per_launch": {"c2_llada_l768": 12959744, "c5_llada_l4096": 68264192}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
-                     "sha256": "8b9b93fb78eb526dd48d92e6b73050e6a46dcac25c98baaf4c4c32f7162da1d1",
-                     "bytes_per_launch": {"c4_llada_l2048": 51188992, "c5_llada_l4096": 116217856}},
+                     "sha256": "5904bb11f13265705d4e4f6ec7dd6af483762e10fe0d7d597d0c44524eb63616",
+                     "bytes_per_launch": {"c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
     "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
                      "sha256": "f7350fa75a2ea8d82120fbfb3ea587e366e2a8716e4a2a11e71f8f323e1ef9f3",
                      "bytes_per_launch": {"c5_llada_l4096_b8": 65324032}},
