@@ -16,7 +16,12 @@
 //            only then the column maxima are reduced (integer warp reductions + shared memory), m is raised,
 //            and O^T and the partial row sums are rescaled.  Row sums are kept per thread (sum over its own
 //            keys) and reduced across the CTA once, at the end;
-//   grid     (C, B*H_kv) as clusters of C in {1, 2, 4, 8} CTAs that split one head's 128-key tiles;
+//   grid     (C, B*H_kv*n_sub) as clusters of C in {1, 2, 4, 8} CTAs that split one head's 128-key tiles.  With
+//            grouped-query attention the g = H_q/H_kv query heads of a kv head are packed into the N axis; when
+//            n*g exceeds the 64 slots the heads are spread over n_sub CTA columns (each takes g/n_sub heads and
+//            streams the same K/V, which the other columns' reads keep in L2).  Every column refreshes the rows of
+//            its key range itself: the columns of a kv head write identical bytes, and each orders its own copy
+//            before its own TMA reads, so whichever copy a read observes holds the fresh row;
 //   refresh  as in the row-major skip kernel: a CTA refreshes the cache rows of its own key range, visits its
 //            tiles in rotated order and waits for the copy only before the first tile that holds one;
 //   merge    CTA c of the cluster owns the output columns d in [c*128/C, (c+1)*128/C): every CTA sends that
@@ -97,7 +102,10 @@ struct KeysParams {
     const int32_t* active_idx;    // nullptr: identity
     __nv_bfloat16* out;
     int32_t* dev_status;
-    int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
+    int n_active, ctx_len, n_q_heads, n_kv_heads;
+    int group;        // query heads of one kv head handled by one CTA column (a divisor of H_q / H_kv)
+    int n_sub;        // CTA columns per kv head = (H_q / H_kv) / group
+    int rows_total;   // n_active * group: packed query rows of one CTA
     int n_splits, tiles_per_split, n_stages;
     int q_tma;                    // 1: the producer fetches Q with one TMA box (MHA); 0: the softmax warps stage it
     uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0
@@ -131,8 +139,9 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     auto bar = [&](int idx) { return bars + idx * 8; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int split = blockIdx.x, bh = blockIdx.y;
+    const int split = blockIdx.x, bh = blockIdx.y / p.n_sub, sub = blockIdx.y % p.n_sub;
     const int b = bh / p.n_kv_heads, hk = bh % p.n_kv_heads;
+    const int hq0 = (hk * p.n_sub + sub) * p.group;        // first query head of this CTA
     const int C = p.n_splits;
     const int DL = HD / C;                                 // output columns this CTA merges
     const int n_tiles_total = (p.ctx_len + BK - 1) / BK;
@@ -181,7 +190,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (lane == 0) {
             if (p.q_tma) {   // Q first: [half][row][64 columns] of this head's rows, rows past n_active read as zero
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
-                tma_load_5d(base, &map_q, 0, 0, hk, 0, b, bar(B_QFULL));
+                tma_load_5d(base, &map_q, 0, 0, hq0, 0, b, bar(B_QFULL));
             }
             int first_tile = 0, j_refreshed = T;
             if (refresh) {
@@ -289,7 +298,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             if (row < p.rows_total) {
                 const int i = row / p.group, jh = row % p.group;
                 v = __ldg(reinterpret_cast<const uint4*>(
-                    p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + ch * 8));
+                    p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + ch * 8));
             }
             const uint32_t off = (ch >> 3) * QHALF + (row >> 3) * 1024 + (row & 7) * 128 + (((ch & 7) ^ (row & 7)) << 4);
             *reinterpret_cast<uint4*>(gbase + off) = v;
@@ -470,7 +479,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             for (int c = 0; c < N; ++c) {
                 if (c < p.rows_total) {
                     const int i = c / p.group, jh = c % p.group;
-                    __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD;
+                    __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD;
                     dst[kk] = __float2bfloat16_rn(__uint_as_float(o[c]) / sh->factor[c]);
                 }
             }
@@ -516,7 +525,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             const float inv = 1.f / l;
             for (int s = 0; s < C; ++s) wgt[s * N + tid] = fast_exp2(recv[s * cf + DL * NP + tid] - m) * inv;
             const int i = tid / p.group, jh = tid % p.group;
-            qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + split * DL;
+            qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL;
         }
         __syncthreads();
         // a thread owns two adjacent output columns of a query row: one 4-byte store
@@ -593,6 +602,7 @@ bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_
 }
 
 struct KeysPlan {
+    int group, n_sub;   // query heads per CTA column, CTA columns per kv head
     int n_slots, n_splits, tiles_per_split, n_stages;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
 };
@@ -601,10 +611,16 @@ constexpr uint32_t kSmemMax = 232448;   // 227 KB: largest dynamic allocation of
 
 KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
     KeysPlan pl{};
-    const int rows = n_active * (d.n_q_heads / d.n_kv_heads);
+    // a CTA column takes the largest divisor of the H_q / H_kv heads of a kv head whose packed rows fit the 64
+    // query slots; the other columns of that kv head stream the same K/V (from L2) for their own heads
+    const int g = d.n_q_heads / d.n_kv_heads;
+    pl.group = g;
+    while (pl.group > 1 && (g % pl.group != 0 || (long long)n_active * pl.group > kMaxRowsT)) --pl.group;
+    pl.n_sub = g / pl.group;
+    const int rows = n_active * pl.group;
     pl.n_slots = rows <= 48 ? 48 : 64;
     const int key_tiles = (d.ctx_len + BK - 1) / BK;
-    const int bh = d.batch * d.n_kv_heads;
+    const int bh = d.batch * d.n_kv_heads * pl.n_sub;
     // one CTA per SM; the cluster size divides the 128 output columns, every CTA gets at least one tile
     int c = 1;
     while (c < 8 && 2 * c * bh <= sm_count() && 2 * c <= key_tiles) c *= 2;
@@ -666,13 +682,12 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
 
 bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
-    const long long rows = (long long)n_active * (d.n_q_heads / d.n_kv_heads);
-    if (rows > kMaxRowsT || n_active > kMaxRowsT) return false;
-    if ((long long)d.batch * d.n_kv_heads > 65535) return false;   // grid.y
+    if (n_active > kMaxRowsT) return false;
     const KeysPlan pl = make_keys_plan(d, n_active);
+    if ((long long)d.batch * d.n_kv_heads * pl.n_sub > 65535) return false;   // grid.y
     // the exchange areas (row-sum scratch, staging, receive buffer) reuse the memory below the refresh list
     // one CTA per SM: beyond one wave of CTAs the row-major skip kernel (two CTAs per SM) streams better
-    if ((long long)pl.n_splits * d.batch * d.n_kv_heads > sm_count()) return false;
+    if ((long long)pl.n_splits * d.batch * d.n_kv_heads * pl.n_sub > sm_count()) return false;
     return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && kRecvOff + kExchangeMax <= pl.off_list;
 }
 
@@ -699,7 +714,8 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.ctx_len = a.d.ctx_len;
     p.n_q_heads = a.d.n_q_heads;
     p.n_kv_heads = a.d.n_kv_heads;
-    p.group = a.d.n_q_heads / a.d.n_kv_heads;
+    p.group = pl.group;
+    p.n_sub = pl.n_sub;
     p.rows_total = a.n_active * p.group;
     p.n_splits = pl.n_splits;
     p.tiles_per_split = pl.tiles_per_split;
@@ -709,8 +725,8 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.off_list = pl.off_list;
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
-    return pl.n_slots == 48 ? launch_n<48>(pl, p, map_k, map_v, map_q, bh, stream)
-                            : launch_n<64>(pl, p, map_k, map_v, map_q, bh, stream);
+    return pl.n_slots == 48 ? launch_n<48>(pl, p, map_k, map_v, map_q, bh * pl.n_sub, stream)
+                            : launch_n<64>(pl, p, map_k, map_v, map_q, bh * pl.n_sub, stream);
 }
 
 }  // namespace ec

@@ -151,6 +151,18 @@ def test_few_row_skip_steps_through_both_slot_counts(Hq, Hkv, n, L):
     _check(w, t, refresh=False)
 
 
+@pytest.mark.parametrize("Hq,Hkv,n,L", [(28, 4, 34, 768), (12, 2, 20, 900), (8, 2, 64, 384), (14, 2, 10, 1500)])
+def test_grouped_query_skip_steps_spread_over_head_columns(Hq, Hkv, n, L):
+    """GQA skip steps whose n x H_q/H_kv packed rows exceed the 64 query slots: the query heads of a kv head are
+    spread over several CTA columns (7 x 1 head at the Dream geometry, 2 x 3, 4 x 1, 1 x 7 heads here), each of
+    which refreshes the same cache rows with the same bytes before reading them."""
+    w = syn.Workload(95, "gqa_columns", syn.BF16, 2, Hq, Hkv, 128, 0, L, 1, 0, 64)
+    idx = syn.arbitrary_active_idx(2, L, n, seed=11 * L + n)
+    t = syn.attn_inputs(w, n, active_idx=idx, std_qk=0.7, std_v=0.5)
+    _check(w, t)
+    _check(w, t, refresh=False)
+
+
 def test_few_row_skip_step_with_rising_maxima():
     """Keys ordered so that the row maxima keep rising from tile to tile (scores grow with the position): the
     lazily updated references must be raised, and the accumulator rescaled, several times."""
