@@ -117,7 +117,8 @@ struct alignas(16) KeysShared {
     uint32_t tmem;
     int abort_flag;
     int n_mine;       // entries of the refresh list
-    int first_tile;   // rotation: the CTA visits its tiles in the order (first_tile + j) mod T
+    int spec_ok;      // 1: the first tile of the range, loaded before the list was known, holds no refreshed row
+    int first_tile;   // rotation of the visiting order, see tile_of()
     int j_refreshed;  // first visit index j whose tile holds a refreshed position (T if none)
     alignas(16) float m[kMaxRowsT];        // reference maxima of the query rows, log2 units (read as float2)
     alignas(16) float factor[kMaxRowsT];   // rescale factors of the current slow path; the row sums at the end
@@ -165,6 +166,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         }
         sh->abort_flag = 0;
         sh->n_mine = 0;
+        sh->spec_ok = 1;
         sh->first_tile = 0;
         sh->j_refreshed = T;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -184,6 +186,14 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     pdl_launch_dependents();
 
     const int key_lo = t_begin * BK, key_hi = min(p.ctx_len, t_end * BK);
+    // Visiting order of the CTA's T tiles.  The producer loads the first tile of the range at once, before the
+    // refresh list is known.  If that tile holds no refreshed row (spec_ok) it is visit 0 and the other tiles
+    // follow in rotated order, those without refreshed rows first; otherwise its data are discarded (that stage
+    // is simply filled again later) and all T tiles are visited in rotated order, shifted by one stage.
+    auto tile_of = [&](int j, int spec_ok, int rot) {
+        if (spec_ok) return j == 0 ? 0 : 1 + (rot + j - 1) % (T - 1);
+        return (rot + j) % T;
+    };
 
     if (warp == 0) {
         // ================================ TMA producer ======================================
@@ -192,27 +202,50 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
                 tma_load_5d(base, &map_q, 0, 0, hq0, 0, b, bar(B_QFULL));
             }
-            int first_tile = 0, j_refreshed = T;
+            auto load_tile = [&](int tile, int stage) {
+                const int key0 = (t_begin + tile) * BK;
+                const uint32_t dst = base + p.off_stage + stage * STAGE;
+                mbar_expect_tx(bar(B_FULL + stage), STAGE);
+                tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + stage));
+                tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + stage));
+            };
+            int spec_ok = 1, rot = 0, j_refreshed = T;
+            load_tile(0, 0);   // visit 0 if it turns out to hold no refreshed row
             if (refresh) {
                 mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
-                first_tile = sh->first_tile;
+                spec_ok = sh->spec_ok;
+                rot = sh->first_tile;
                 j_refreshed = sh->j_refreshed;
             }
-            for (int j = 0; j < T; ++j) {
-                const int s = j % NS, u = j / NS;
-                int tile = first_tile + j;
-                if (tile >= T) tile -= T;
-                const int key0 = (t_begin + tile) * BK;
+            const int soff = spec_ok ? 0 : 1;   // stage shift: the discarded fill took stage 0's first phase
+            bool discard_seen = spec_ok != 0;
+            for (int j = spec_ok ? 1 : 0; j < T; ++j) {
+                const int s = (j + soff) % NS, u = (j + soff) / NS;
                 if (j == j_refreshed) mbar_wait(bar(B_REFRESHED), 0, abort_flag, p.dev_status);
-                if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
-                const uint32_t dst = base + p.off_stage + s * STAGE;
-                mbar_expect_tx(bar(B_FULL + s), STAGE);
-                tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
-                tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
+                if (u > 0) {
+                    if (soff == 1 && s == 0) {
+                        // stage 0: its phase 0 was the discarded fill, which nobody consumes or releases
+                        if (u == 1) {
+                            mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);
+                            discard_seen = true;
+                        } else {
+                            mbar_wait(bar(B_EMPTY + 0), (u - 2) & 1, abort_flag, p.dev_status);
+                        }
+                    } else {
+                        mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
+                    }
+                }
+                load_tile(tile_of(j, spec_ok, rot), s);
             }
+            if (!discard_seen) mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);   // no copy in flight at exit
+        }
+        if (C > 1) {   // this warp no longer touches the memory the peers' partials will land in
+            __syncwarp();
+            cluster_arrive();
         }
     } else if (warp == 1) {
         // ================= refresh list, then MMA issue (lane 0) =================================
+        bool spec_ok_w1 = true;
         if (refresh) {
             int posv[kMaxRowsT / 32];
 #pragma unroll
@@ -221,7 +254,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 posv[k] = -1;
                 if (i < p.n_active) posv[k] = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
             }
-            int n_mine = 0, hi_tile = -1;   // hi_tile: last local tile that holds a refreshed position
+            int n_mine = 0, hi_tile = -1, lo_tile = T;   // last / first local tile that holds a refreshed position
 #pragma unroll
             for (int k = 0; k < kMaxRowsT / 32; ++k) {
                 const bool hit = posv[k] >= key_lo && posv[k] < key_hi;
@@ -229,17 +262,29 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 if (hit) {
                     list[n_mine + __popc(mk & ((1u << lane) - 1u))] = make_int2(k * 32 + lane, posv[k]);
                     hi_tile = max(hi_tile, (posv[k] - key_lo) / BK);
+                    lo_tile = min(lo_tile, (posv[k] - key_lo) / BK);
                 }
                 n_mine += __popc(mk);
             }
             hi_tile = __reduce_max_sync(0xffffffffu, hi_tile);
-            const int first_tile = n_mine > 0 ? (hi_tile + 1) % T : 0;
+            lo_tile = __reduce_min_sync(0xffffffffu, lo_tile);
+            spec_ok_w1 = lo_tile > 0;   // the tile loaded ahead of this list holds no refreshed row
+            int rot = 0;
+            if (n_mine > 0) rot = spec_ok_w1 ? hi_tile % (T - 1) : (hi_tile + 1) % T;   // (spec_ok and n_mine > 0 imply T > 1)
             int j_ref = T;
 #pragma unroll
             for (int k = 0; k < kMaxRowsT / 32; ++k) {
                 if (posv[k] >= key_lo && posv[k] < key_hi) {
-                    int j = (posv[k] - key_lo) / BK - first_tile;
-                    if (j < 0) j += T;
+                    const int tile = (posv[k] - key_lo) / BK;
+                    int j;
+                    if (spec_ok_w1) {
+                        j = tile - 1 - rot;
+                        if (j < 0) j += T - 1;
+                        j += 1;
+                    } else {
+                        j = tile - rot;
+                        if (j < 0) j += T;
+                    }
                     j_ref = min(j_ref, j);
                 }
             }
@@ -247,7 +292,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             __syncwarp();
             if (lane == 0) {
                 sh->n_mine = n_mine;
-                sh->first_tile = first_tile;
+                sh->spec_ok = spec_ok_w1 ? 1 : 0;
+                sh->first_tile = rot;
                 sh->j_refreshed = j_ref;
                 mbar_arrive(bar(B_LIST));
             }
@@ -256,8 +302,11 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             constexpr uint32_t IDESC_S = instr_desc2(N, 0, 0);    // A = K tile (K-major), B = Q (K-major)
             constexpr uint32_t IDESC_PV = instr_desc2(N, 1, 1);   // A = V tile (MN-major: d contiguous), B = P^T (MN-major)
             constexpr uint32_t QHALF = N * 128;                   // bytes of one 64-column half of the Q tile
+            const int soff = spec_ok_w1 ? 0 : 1;
+            auto stage_of = [&](int j) { return (j + soff) % NS; };
+            auto wait_stage = [&](int j) { mbar_wait(bar(B_FULL + stage_of(j)), ((j + soff) / NS) & 1, abort_flag, p.dev_status); };
             auto issue_s = [&](int j) {
-                const uint32_t kst = base + p.off_stage + (j % NS) * STAGE;
+                const uint32_t kst = base + p.off_stage + stage_of(j) * STAGE;
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t koff = (k & 3) * 32;
@@ -267,16 +316,16 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 commit(bar(B_SFULL + (j & 1)));
             };
             mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
-            mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);
+            wait_stage(0);
             fence_after();
             issue_s(0);
             for (int j = 0; j < T; ++j) {
                 if (j + 1 < T) {
-                    mbar_wait(bar(B_FULL + (j + 1) % NS), ((j + 1) / NS) & 1, abort_flag, p.dev_status);
+                    wait_stage(j + 1);
                     fence_after();
                     issue_s(j + 1);
                 }
-                const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + TILE;
+                const uint32_t vst = base + p.off_stage + stage_of(j) * STAGE + TILE;
                 mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
                 fence_after();
 #pragma unroll
@@ -284,8 +333,12 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                     mma_ss(tmem + TM_O, smem_desc(vst + k * 2048, SUB, 1024), smem_desc(base + p.off_p + k * 2048, SUB, 1024),
                            IDESC_PV, (j > 0 || k > 0));
                 commit(bar(B_PVDONE));
-                commit(bar(B_EMPTY + j % NS));
+                commit(bar(B_EMPTY + stage_of(j)));
             }
+        }
+        if (C > 1) {   // (the products still in flight are covered by the softmax warps, which arrive after the last one)
+            __syncwarp();
+            cluster_arrive();
         }
     } else {
         // ================== Q staging, cache refresh, softmax (warps 2..5) ========================
@@ -308,10 +361,11 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             mbar_arrive(bar(B_QFULL));
         }
 
-        int first_tile = 0;
+        int spec_ok = 1, rot = 0;
         if (refresh) {
             mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
-            first_tile = sh->first_tile;
+            spec_ok = sh->spec_ok;
+            rot = sh->first_tile;
             // fresh rows of this CTA's key range -> cache in global memory, eight 16-byte pieces in flight per thread
             const int chunks = sh->n_mine * 32;
             for (int c0 = stid; c0 < chunks; c0 += 8 * kSoft) {
@@ -360,9 +414,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             ld32(s_addr, sr);
             if (N == 48) ld16(s_addr + 32, sr + 32); else ld32(s_addr + 32, sr + 32);
             wait_ld();
-            int tile = first_tile + j;
-            if (tile >= T) tile -= T;
-            const int key = (t_begin + tile) * BK + kk;
+            const int key = (t_begin + tile_of(j, spec_ok, rot)) * BK + kk;
             if (key >= p.ctx_len) {   // only in the ragged last tile of the context
 #pragma unroll
                 for (int c = 0; c < N; ++c) sr[c] = 0xff800000u;   // -inf: probability 0 for every query
@@ -440,6 +492,12 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         }
         mbar_wait(bar(B_PVDONE), (T - 1) & 1, abort_flag, p.dev_status);   // Q, P^T and the K/V stages are dead from here on
         fence_after();
+        if (C > 1) {
+            // first cluster barrier, arrive half: from here on the peers may write their partials into this CTA's
+            // receive buffer (dead stage memory that the reduction and the staging below do not touch)
+            __syncwarp();
+            cluster_arrive();
+        }
 
         // ---- row sums over the CTA's keys: per-thread partials -> shared memory -> one thread per query ----
         float* lred = reinterpret_cast<float*>(gbase);   // [128 keys][NP]
@@ -501,10 +559,9 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     }
 
     if (C > 1) {
-        // every CTA of the cluster is past its main loop (its Q, P^T and K/V stages are dead, its barriers
-        // initialised) and has staged its slices
-        __syncwarp();
-        cluster_arrive();
+        // the slices are staged (CTA barrier: the softmax warps wrote them, warp 0 sends them) and every CTA of
+        // the cluster is past its main loop (its Q, P^T and K/V stages are dead, its barriers initialised)
+        __syncthreads();
         cluster_wait();
         if (warp == 0 && lane < C) {   // one bulk copy per owner into the owner's receive buffer
             const uint32_t src = base + kStagingOff + (uint32_t)lane * chunk_bytes;
@@ -513,6 +570,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         }
         // ---- merge the C partials of the output columns this CTA owns -------------------------
         mbar_wait(bar(B_RECV), 0, abort_flag, p.dev_status);
+        // second cluster barrier, arrive half: this CTA holds every peer's partial, i.e. the peers' copies out of
+        // their staging areas have completed; the wait half, before leaving, overlaps the merge
+        __syncwarp();
+        cluster_arrive();
         const float* recv = reinterpret_cast<const float*>(gbase + kRecvOff);
         const int cf = (int)(chunk_bytes / 4);
         float* wgt = reinterpret_cast<float*>(gbase);   // [C][N] normalised weights 2^(m_s - m) / l, over the dead row-sum scratch
@@ -542,7 +603,6 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         }
         // no CTA leaves while a peer may still copy out of or into its shared memory
         __syncwarp();
-        cluster_arrive();
         cluster_wait();
     }
 
