@@ -408,28 +408,66 @@ def run_cuda(args) -> None:
     ms_refresh = _graph_time(torch, refresh_only_skip, reps, 3, stream) / n_layers
 
     # ---- end to end through the binding with host buffers --------------------------
+    # Per step every layer's q / k_new / v_new come from pinned host memory and every layer's output goes back, as do
+    # the step's logits and the gate's decision.  The layers' inputs sit back to back in one host arena and one device
+    # arena (the tensors the library sees are views), so a group of layers moves with ONE copy; inputs go up on one
+    # copy stream, results come back on another, the kernels run on the compute stream, and events order a group's
+    # kernels after its inputs and its read-back after its kernels: PCIe traffic in both directions overlaps the
+    # kernels of the neighbouring groups.
     dt = torch.bfloat16 if w.dtype == syn.BF16 else torch.float32
-    hq = [t.cpu().pin_memory() for t in wl.q_s]
-    hk = [t.cpu().pin_memory() for t in wl.kn_s]
-    hv = [t.cpu().pin_memory() for t in wl.vn_s]
+    nq, nkv = wl.q_s[0].numel(), wl.kn_s[0].numel()
+    per_layer = nq + 2 * nkv
+    in_dev = torch.empty(n_layers * per_layer, device=dev, dtype=dt)
+    in_host = torch.empty(n_layers * per_layer, dtype=dt).pin_memory()
+    out_dev = torch.empty(n_layers * nq, device=dev, dtype=dt)
+    out_host = torch.empty(n_layers * nq, dtype=dt).pin_memory()
+    q_e, k_e, v_e, o_e = [], [], [], []
+    for l in range(n_layers):
+        o = l * per_layer
+        q_e.append(in_dev[o:o + nq].view(wl.q_s[l].shape))
+        k_e.append(in_dev[o + nq:o + nq + nkv].view(wl.kn_s[l].shape))
+        v_e.append(in_dev[o + nq + nkv:o + per_layer].view(wl.vn_s[l].shape))
+        o_e.append(out_dev[l * nq:(l + 1) * nq].view(wl.q_s[l].shape))
+        in_host[o:o + nq].copy_(wl.q_s[l].reshape(-1).cpu())
+        in_host[o + nq:o + nq + nkv].copy_(wl.kn_s[l].reshape(-1).cpu())
+        in_host[o + nq + nkv:o + per_layer].copy_(wl.vn_s[l].reshape(-1).cpu())
     hlog = wl.logits[0].cpu().pin_memory()
-    hout = [torch.empty_like(t, device="cpu").pin_memory() for t in wl.out_s]
     hdec = torch.empty_like(wl.dec, device="cpu").pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in hq + hk + hv) + hlog.numel() * hlog.element_size()
-    d2h = sum(t.numel() * t.element_size() for t in hout) + hdec.numel() * hdec.element_size()
+    h2d = in_host.numel() * in_host.element_size() + hlog.numel() * hlog.element_size()
+    d2h = out_host.numel() * out_host.element_size() + hdec.numel() * hdec.element_size()
+    group = 4 if n_layers >= 8 else 1
+    groups = [(g0, min(n_layers, g0 + group)) for g0 in range(0, n_layers, group)]
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(len(groups) + 1)]
+    ev_done = [torch.cuda.Event() for _ in range(len(groups) + 1)]
 
     def e2e_step():
-        with torch.cuda.stream(stream):
-            for l in range(n_layers):
-                wl.q_s[l].copy_(hq[l], non_blocking=True)
-                wl.kn_s[l].copy_(hk[l], non_blocking=True)
-                wl.vn_s[l].copy_(hv[l], non_blocking=True)
-                wl.attend_skip(l)
-                hout[l].copy_(wl.out_s[l], non_blocking=True)
+        with torch.cuda.stream(s_in):
+            for gi, (l0, l1) in enumerate(groups):
+                in_dev[l0 * per_layer:l1 * per_layer].copy_(in_host[l0 * per_layer:l1 * per_layer], non_blocking=True)
+                ev_in[gi].record(s_in)
             wl.logits[0].copy_(hlog, non_blocking=True)
+            ev_in[-1].record(s_in)
+        for gi, (l0, l1) in enumerate(groups):
+            stream.wait_event(ev_in[gi])
+            with torch.cuda.stream(stream):
+                for l in range(l0, l1):
+                    ec.ec_attend(wl.desc, q_e[l], k_e[l], v_e[l], wl.k_cache[l], wl.v_cache[l], wl.idx, out=o_e[l],
+                                 workspace=wl.ws_s)
+            ev_done[gi].record(stream)
+            s_out.wait_event(ev_done[gi])
+            with torch.cuda.stream(s_out):
+                out_host[l0 * nq:l1 * nq].copy_(out_dev[l0 * nq:l1 * nq], non_blocking=True)
+        stream.wait_event(ev_in[-1])
+        with torch.cuda.stream(stream):
             wl.gate(0)
+        ev_done[-1].record(stream)
+        s_out.wait_event(ev_done[-1])
+        with torch.cuda.stream(s_out):
             hdec.copy_(wl.dec, non_blocking=True)
-        stream.synchronize()  # the host reads the decision to choose the next step's path
+        s_out.synchronize()   # the host reads the decision to choose the next step's path ...
+        stream.synchronize()  # ... and every stream is idle before the next step reuses the buffers
+        s_in.synchronize()
 
     for _ in range(3):
         e2e_step()
