@@ -8,7 +8,9 @@ bf16 bit patterns (dtype 0 / 1).
 
 Passages followed: Section 4.2 and Appendix A (partial step: refresh the active
 rows' K/V, attend from the active rows over every position), Eq. 1 and
-Algorithm 1 (entropy of each decoded row, maximum, comparison with tau).
+Algorithm 1 (entropy of each decoded row, maximum, comparison with tau), Eq. 2-3 and
+Appendix A (decode history, recent-token selection, skip_flag / dt bookkeeping; plain
+numpy at the end of this file).
 """
 from __future__ import annotations
 
@@ -148,3 +150,47 @@ def entropy_gate(logits: np.ndarray, dtype: int, vocab: int, decoded_flags: np.n
     if rc:
         raise ValueError("oracle_entropy_gate: n_rows must be a multiple of rows_per_seq")
     return dict(argmax=argmax, conf=conf, entropy=ent, max_entropy=maxh, decision=dec, probs=probs)
+
+
+# --------------------------------------------------------------------------- #
+# Recent-token selection and the per-step bookkeeping (Eq. 2-3, Appendix A).
+# Plain numpy on float64 histories with -inf for "never decoded".
+# --------------------------------------------------------------------------- #
+def select_recent(H: np.ndarray, k: int, t: int, dt: int) -> np.ndarray:
+    """Eq. 3.  H is the decode history of Eq. 2 (H_i = step at which position i was decoded, -inf otherwise).
+    K = a set of k positions with the largest sum of H, i.e. the k largest entries; tau_R = max(min over K of H,
+    t - dt); returns the positions of R = {i : H_i >= tau_R} in ascending order.  With fewer than k decoded
+    positions K has to contain never-decoded ones, so its minimum is -inf and tau_R = t - dt; k = 0 leaves
+    the minimum over an empty set, +inf, so R is empty.  Ties at the threshold all belong to R (|R| may exceed k)."""
+    H = np.asarray(H, dtype=np.float64)
+    if k < 0 or k > H.size:
+        raise ValueError("k must lie in [0, len(H)]")
+    if k == 0:
+        min_k = np.inf
+    else:
+        min_k = np.sort(H)[::-1][k - 1]          # the k-th largest entry = min over the top-k set
+    tau_r = max(min_k, float(t - dt))
+    return np.flatnonzero(H >= tau_r).astype(np.int64)
+
+
+def step_bookkeeping(H: np.ndarray, t: int, dt: int, decoded_pos, decision: int, k: int):
+    """Appendix A, the statements after the decode of step t, in the paper's order:
+        H[D] <- t;  K, tau_R, R as in Eq. 3 (with the t and dt of THIS step);
+        E <= tau  =>  skip_flag <- True,  dt <- dt + 1;   else  skip_flag <- False, dt <- 0;   t <- t + 1.
+    `decision` is the gate's verdict (SKIP = 0: E <= tau, RECOMPUTE = 1).  H is updated in place.
+    Returns (R, skip_flag, dt_next, t_next)."""
+    H[np.asarray(decoded_pos, dtype=np.int64)] = float(t)
+    R = select_recent(H, k, t, dt)
+    skip_flag = decision == SKIP
+    dt_next = dt + 1 if skip_flag else 0
+    return R, skip_flag, dt_next, t + 1
+
+
+def partial_step_rows(window_start: int, block: int, R: np.ndarray) -> np.ndarray:
+    """Active rows of a partial step: the positions of the current block (the mask tokens' block), then the
+    recent positions outside it, ascending.  (Appendix A: the rows M u R of the partial branch; the block is
+    taken whole, which keeps the row count of a step fixed at block + |R outside the block|.)"""
+    window = np.arange(window_start, window_start + block, dtype=np.int64)
+    R = np.asarray(R, dtype=np.int64)
+    outside = R[(R < window_start) | (R >= window_start + block)]
+    return np.concatenate([window, np.sort(outside)])

@@ -51,13 +51,15 @@ class ReplayState:
         return np.concatenate([window, rec]).astype(np.int32)
 
     def record(self, decoded_rows: np.ndarray, decision: int) -> None:
-        """decode-history update, then the gate's verdict (Appendix A, end of the loop body)."""
-        self.t += 1
+        """decode-history update with the step's own index, then the gate's verdict, then t <- t + 1 (Appendix A,
+        end of the loop body).  The recent set is formed at the start of the next step from (t + 1) - (dt + 1) =
+        t - dt, the value Appendix A uses when it selects right after the decode."""
         pos = self.block_start + np.flatnonzero(decoded_rows)
         self.H[pos] = self.t
         self.masked[np.flatnonzero(decoded_rows)] = False
         self.skip_flag = decision == 0
         self.dt = self.dt + 1 if self.skip_flag else 0
+        self.t += 1
 
 
 def step_inputs(w: syn.Workload, step: int, n_active: int, sigma_centre: float | None = None) -> dict:

@@ -415,3 +415,78 @@ def test_identity_refresh_is_a_transposed_copy():
     oracle.kv_refresh(k, v, t["k_new"], t["v_new"], None, syn.BF16)
     assert np.array_equal(k, np.transpose(t["k_new"], (0, 2, 1, 3)))
     assert np.array_equal(v, np.transpose(t["v_new"], (0, 2, 1, 3)))
+
+
+# --------------------------------------------------------------------------- #
+# Recent-token selection (Eq. 2-3) and the step bookkeeping of Appendix A
+# --------------------------------------------------------------------------- #
+def _parse_h(s):
+    return np.array([-np.inf if x.strip() == "n" else float(x) for x in s.split(",")])
+
+
+def test_recent_selection_matches_the_hand_worked_cases():
+    path = os.path.join(os.path.dirname(__file__), "golden", "recent_selection_worked.txt")
+    n = 0
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        h, k, t, dt, exp = [x.strip() for x in line.split("|")]
+        want = [int(x) for x in exp.split(",")] if exp else []
+        got = oracle.select_recent(_parse_h(h), int(k), int(t), int(dt)).tolist()
+        assert got == want, line
+        n += 1
+    assert n >= 9
+
+
+def test_recent_selection_threshold_equals_brute_force_over_all_k_subsets():
+    """Eq. 3 literally: K maximises the sum of H over all subsets of size k (never-decoded entries count as a very
+    negative number so that they are taken last); the minimum over K is unique even when K is not."""
+    import itertools
+
+    rng = np.random.Generator(np.random.PCG64(31))
+    for trial in range(60):
+        n = int(rng.integers(3, 9))
+        H = rng.integers(0, 5, size=n).astype(np.float64)
+        H[rng.random(n) < 0.35] = -np.inf
+        k = int(rng.integers(1, n + 1))
+        t, dt = 5, int(rng.integers(0, 6))
+        big = np.where(np.isfinite(H), H, -1e9)
+        best = max(itertools.combinations(range(n), k), key=lambda s: sum(big[list(s)]))
+        min_k = min(H[list(best)])
+        tau_r = max(min_k, t - dt)
+        want = [i for i in range(n) if H[i] >= tau_r]
+        assert oracle.select_recent(H, k, t, dt).tolist() == want
+
+
+def test_recent_selection_properties():
+    rng = np.random.Generator(np.random.PCG64(32))
+    H = rng.integers(1, 40, size=300).astype(np.float64)
+    H[rng.random(300) < 0.5] = -np.inf
+    t = 40
+    assert oracle.select_recent(H, 0, t, 10).size == 0                       # no budget, nothing selected
+    prev = -1
+    for k in (1, 2, 8, 64, 150, 300):                                         # a larger budget never selects less
+        R = oracle.select_recent(H, k, t, 40)
+        assert R.size >= min(k, int(np.isfinite(H).sum())) and R.size >= prev
+        assert np.all(np.diff(R) > 0) and np.all(np.isfinite(H[R]))
+        prev = R.size
+    for dt in range(0, 12):                                                   # never older than the last full pass
+        R = oracle.select_recent(H, 64, t, dt)
+        assert np.all(H[R] >= t - dt)
+    R0 = oracle.select_recent(H, 64, t, 0)
+    assert set(R0.tolist()) == set(np.flatnonzero(H == t).tolist())          # dt = 0: only this step's tokens
+
+
+def test_step_bookkeeping_follows_appendix_a_order():
+    H = np.full(12, -np.inf)
+    # step t = 1 (a full pass happened, dt = 0): positions 4, 5 decoded, gate says skip
+    R, skip, dt, t = oracle.step_bookkeeping(H, 1, 0, [4, 5], oracle.SKIP, k=2)
+    assert H[4] == 1 and H[5] == 1 and R.tolist() == [4, 5] and skip and dt == 1 and t == 2
+    # step 2 (partial), position 6 decoded, gate says skip: K = {6, one of 4/5}, min 1, tau_R = max(1, 2 - 1) = 1
+    R, skip, dt, t = oracle.step_bookkeeping(H, t, dt, [6], oracle.SKIP, k=2)
+    assert R.tolist() == [4, 5, 6] and dt == 2 and t == 3
+    # step 3, position 7 decoded, gate says recompute: the selection still uses dt = 2 (tau_R = max(2, 1) = 2)
+    R, skip, dt, t = oracle.step_bookkeeping(H, t, dt, [7], oracle.RECOMPUTE, k=2)
+    assert R.tolist() == [6, 7] and not skip and dt == 0 and t == 4
+    rows = oracle.partial_step_rows(4, 4, np.array([1, 5, 9, 6]))
+    assert rows.tolist() == [4, 5, 6, 7, 1, 9]
