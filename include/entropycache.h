@@ -13,6 +13,11 @@
  *                    confidence, Shannon entropy), maximum entropy over the
  *                    newly decoded rows, comparison with tau   (Eq. 1; Algorithm 1)
  *
+ * and one keeps the loop's state on the device between steps:
+ *
+ *   ec_select_recent decode history, recent-token set R, skip_flag / dt bookkeeping and
+ *                    the next partial step's row list          (Eq. 2-3; Appendix A)
+ *
  * "Active rows" are the mask tokens of the current block/window plus the k most
  * recently decoded tokens (M u R); on a recompute step every row is active.
  *
@@ -155,6 +160,39 @@ ec_status ec_entropy_gate_static(const void *logits, int32_t dtype, int32_t n_ro
                                  const uint8_t *decoded_flags, float tau,
                                  int32_t *argmax_out, float *conf_out, float *entropy_out,
                                  float *max_entropy_out, int32_t *decision_out, void *stream);
+
+/* Eq. 2: history value of a position that has not been decoded ("-infinity"). */
+#define EC_H_NEVER INT32_MIN
+
+/* Per-sequence state of the cached denoising loop (Algorithm 1; Appendix A), DEVICE memory,
+ * one element per sequence; the caller initialises it (t = first step index, the rest 0). */
+typedef struct {
+    int32_t t;             /* index of the current time step */
+    int32_t dt_recompute;  /* steps elapsed since the last full recomputation */
+    int32_t skip_flag;     /* 1: the next step is a partial step (the gate said E <= tau) */
+    int32_t n_active;      /* out: rows of the next partial step (may exceed n_cap, see below) */
+} ec_step_state;
+
+/* Eq. 2-3 and the bookkeeping of Appendix A after the decode of step t, for `batch`
+ * sequences in one launch, in the paper's order:
+ *   1. history[b, window_start[b] + r] = t_b  for every r < block with decoded_flags[b*block + r] != 0   (Eq. 2)
+ *   2. K = the k positions of sequence b with the largest history values; tau_R = max(min over K, t_b - dt_b);
+ *      R = { i : history[b, i] >= tau_R }    (Eq. 3; ties at the threshold all belong to R; with fewer than k
+ *      decoded positions the minimum is "-infinity" and tau_R = t_b - dt_b; k = 0 gives the empty set)
+ *   3. skip_flag_b = (decision[b] == EC_SKIP);  dt_b = skip_flag_b ? dt_b + 1 : 0;  t_b = t_b + 1
+ *   4. active_idx[b, :] = the block's positions window_start[b] .. window_start[b] + block - 1, then the
+ *      positions of R outside the block in ascending order, then -1 up to n_cap (ec_attend and ec_kv_refresh
+ *      skip negative positions); state[b].n_active = block + |R outside the block|.  If that exceeds n_cap the
+ *      list is cut at n_cap entries: the caller compares n_active with n_cap and runs a full step instead.
+ * history: int32 [batch, ctx_len], EC_H_NEVER where nothing was decoded; decoded_flags: uint8 [batch * block]
+ * (the array ec_entropy_gate takes); window_start, decision: int32 [batch]; active_idx: int32 [batch, n_cap].
+ * All DEVICE pointers.  0 <= k <= ctx_len, block <= n_cap, and every window must lie inside [0, ctx_len]:
+ * a window that does not makes the kernel leave that sequence untouched and set its n_active to -1.
+ * ctx_len is limited to 16384 (EC_ERR_UNSUPPORTED beyond). */
+ec_status ec_select_recent(int32_t *history, int32_t ctx_len, int32_t batch, ec_step_state *state,
+                           const uint8_t *decoded_flags, const int32_t *window_start, int32_t block,
+                           const int32_t *decision, int32_t k, int32_t *active_idx, int32_t n_cap,
+                           void *stream);
 
 /* Zero-fills a workspace (asynchronous on `stream`). */
 ec_status ec_workspace_init(void *workspace, size_t workspace_bytes, void *stream);

@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.ec_entropy_gate.restype = i32
     lib.ec_entropy_gate_static.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
     lib.ec_entropy_gate_static.restype = i32
+    lib.ec_select_recent.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, i32, vp, i32, vp]
+    lib.ec_select_recent.restype = i32
     lib.ec_workspace_init.argtypes = [vp, sz, vp]
     lib.ec_workspace_init.restype = i32
     lib.ec_status_string.argtypes = [i32]
@@ -218,3 +220,38 @@ def ec_entropy_gate_static(logits, vocab: int, rows_per_seq: int, decoded_flags,
                                       _dev(entropy_out, "entropy_out"), _dev(max_entropy_out, "max_entropy_out"),
                                       _dev(decision_out, "decision_out"), _stream(stream)),
            "ec_entropy_gate_static")
+
+
+EC_H_NEVER = -(2 ** 31)
+
+
+def new_step_state(batch: int, t0: int = 1, device="cuda") -> torch.Tensor:
+    """int32 [batch, 4] = ec_step_state per sequence: (t, dt_recompute, skip_flag, n_active)."""
+    st = torch.zeros(batch, 4, dtype=torch.int32, device=device)
+    st[:, 0] = t0
+    return st
+
+
+def new_history(batch: int, ctx_len: int, device="cuda") -> torch.Tensor:
+    """int32 [batch, ctx_len] decode history (Eq. 2), every position never decoded."""
+    return torch.full((batch, ctx_len), EC_H_NEVER, dtype=torch.int32, device=device)
+
+
+def ec_select_recent(history, state, decoded_flags, window_start, block: int, decision, k: int, active_idx,
+                     stream=None) -> None:
+    """Eq. 2-3 and the bookkeeping of Appendix A after the decode of a step (argument marshalling only).
+    history int32 [B, L]; state int32 [B, 4]; decoded_flags uint8 [B * block]; window_start, decision int32 [B];
+    active_idx int32 [B, n_cap] (out)."""
+    batch, ctx_len = history.shape
+    if history.dtype != torch.int32 or state.dtype != torch.int32 or active_idx.dtype != torch.int32:
+        raise TypeError("history, state and active_idx must be int32")
+    if decoded_flags.dtype != torch.uint8 or window_start.dtype != torch.int32 or decision.dtype != torch.int32:
+        raise TypeError("decoded_flags must be uint8, window_start and decision int32")
+    if tuple(state.shape) != (batch, 4) or active_idx.shape[0] != batch or decoded_flags.numel() != batch * block:
+        raise ValueError("state must be [B, 4], active_idx [B, n_cap], decoded_flags [B * block]")
+    if window_start.numel() != batch or decision.numel() != batch:
+        raise ValueError("window_start and decision must hold one entry per sequence")
+    _check(lib.ec_select_recent(_dev(history, "history"), int(ctx_len), int(batch), _dev(state, "state"),
+                                _dev(decoded_flags, "decoded_flags"), _dev(window_start, "window_start"), int(block),
+                                _dev(decision, "decision"), int(k), _dev(active_idx, "active_idx"),
+                                int(active_idx.shape[1]), _stream(stream)), "ec_select_recent")

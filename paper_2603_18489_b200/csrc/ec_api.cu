@@ -95,6 +95,18 @@ ec_status ec_kv_refresh(const ec_attn_desc* desc, void* k_cache, void* v_cache, 
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 
+ec_status ec_select_recent(int32_t* history, int32_t ctx_len, int32_t batch, ec_step_state* state,
+                           const uint8_t* decoded_flags, const int32_t* window_start, int32_t block,
+                           const int32_t* decision, int32_t k, int32_t* active_idx, int32_t n_cap, void* stream) {
+    if (!history || !state || !decoded_flags || !window_start || !decision || !active_idx) return EC_ERR_NULL;
+    if (ctx_len < 1 || batch < 1 || block < 1 || block > ctx_len || k < 0 || k > ctx_len || n_cap < block)
+        return EC_ERR_SHAPE;
+    if (ctx_len > select_recent_max_ctx() || batch > 65535) return EC_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_select_recent(history, ctx_len, batch, state, decoded_flags, window_start, block,
+                                               decision, k, active_idx, n_cap, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
 size_t ec_attend_workspace_bytes(const ec_attn_desc* desc, int32_t n_active) {
     if (check_desc(desc) != EC_OK || n_active < 0 || n_active > desc->ctx_len) return 0;
     return attend_ws(*desc, n_active);
