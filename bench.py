@@ -407,6 +407,17 @@ def run_cuda(args) -> None:
     ms_gate = _graph_time(torch, gate_only, reps, 3, stream) / wl.n_lbuf
     ms_refresh = _graph_time(torch, refresh_only_skip, reps, 3, stream) / n_layers
 
+    # the loop's bookkeeping on the device (decode history, recent set, next row list): eight calls per replay
+    sel_hist, sel_state = ec.new_history(w.batch, w.ctx_len, dev), ec.new_step_state(w.batch, 1, dev)
+    sel_idx = torch.empty(w.batch, w.block + 64, dtype=torch.int32, device=dev)
+    sel_w0 = torch.full((w.batch,), w.prompt_len, dtype=torch.int32, device=dev)
+
+    def select_only():
+        for _ in range(8):
+            ec.ec_select_recent(sel_hist, sel_state, wl.flags, sel_w0, w.block, wl.dec, w.k_recent, sel_idx)
+
+    ms_select = _graph_time(torch, select_only, reps, 3, stream) / 8
+
     # ---- end to end through the binding with host buffers --------------------------
     # Per step every layer's q / k_new / v_new come from pinned host memory and every layer's output goes back, as do
     # the step's logits and the gate's decision.  The layers' inputs sit back to back in one host arena and one device
@@ -506,7 +517,8 @@ def run_cuda(args) -> None:
         "recompute": {"us_per_layer_step": us_rec, "ms_per_step": ms_rec,
                       "skip_over_recompute": us_skip / us_rec},
         "kernels_us": {"attend_skip": ms_att_skip * 1e3, "attend_recompute": ms_att_rec * 1e3,
-                       "entropy_gate": ms_gate * 1e3, "kv_refresh_skip": ms_refresh * 1e3},
+                       "entropy_gate": ms_gate * 1e3, "kv_refresh_skip": ms_refresh * 1e3,
+                       "select_recent": ms_select * 1e3},
         "roofline": {"kernel": "ec_attend skip path (one launch: refresh + attention + merge)", "bound": "hbm",
                      "achieved": att_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": att_gbs / peaks["hbm_gbs"], "traffic": _ncu_traffic("attend_skip", w.name),

@@ -82,8 +82,10 @@ typedef struct {
  *   q, out            [batch, n_active,  n_q_heads,  head_dim]   (post-RoPE Q)
  *   active_idx        int32 [batch, n_active]; positions in [0, ctx_len), unique
  *                     within a sequence (duplicates: the surviving row is
- *                     unspecified).  NULL means the identity list 0..ctx_len-1
- *                     and requires n_active == ctx_len (recompute step).
+ *                     unspecified).  An entry outside [0, ctx_len), such as the -1
+ *                     padding ec_select_recent writes, refreshes nothing; its row of
+ *                     `out` is unspecified.  NULL means the identity list
+ *                     0..ctx_len-1 and requires n_active == ctx_len (recompute step).
  */
 
 /* Section 4.2 / Appendix A (partial branch): the active rows get fresh K,V, every

@@ -110,3 +110,71 @@ def test_config4_block_replay_with_drifting_sigma(k):
     n_full = sum(r["full"] for r in ref)
     assert 2 <= n_full <= 12
     assert all(r["n_active"] in (w.ctx_len,) or 32 <= r["n_active"] <= 32 + 32 for r in ref)
+
+
+@pytest.mark.parametrize("name,k,n_steps", [("c1_tiny_fp32", 2, 10), ("c2_llada_l768", 2, 12), ("c2_llada_l768", 6, 12)])
+def test_loop_state_kept_on_the_device(name, k, n_steps):
+    """The whole loop of Appendix A with its state on the GPU: the gate's decision tensor and the step's decoded
+    flags go straight into ec_select_recent, whose row list (padded with -1 up to a fixed capacity) goes straight
+    into ec_attend; the host only reads skip_flag to pick the branch.  Every step is compared with the oracle
+    (attention output of the real rows, E, decision, history, row list); at the end the caches byte for byte."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.WORKLOADS[name]
+    assert w.batch == 1
+    dev = torch.device("cuda")
+    n_cap = w.block + 8
+    tau = _tau_for_recompute_share(w, n_steps, 0.3)
+    kc, vc = _caches(w)
+    okc, ovc = kc.copy(), vc.copy()
+    gk, gv = to_dev(kc), to_dev(vc)
+    d = ec.make_desc(1, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    hist, state = ec.new_history(1, w.ctx_len), ec.new_step_state(1, 1)
+    idx_dev = torch.full((1, n_cap), -1, dtype=torch.int32, device=dev)
+    w0 = w.prompt_len
+    w0_dev = torch.tensor([w0], dtype=torch.int32, device=dev)
+    H, t, dt, skip = np.full(w.ctx_len, -np.inf), 1, 0, False
+    rows = None
+    host = ReplayState(w)          # only for the seeded choice of which rows get decoded
+    n_partial = 0
+    for s in range(n_steps):
+        st = state.cpu().numpy()[0]
+        assert st[0] == t and st[1] == dt and st[2] == int(skip)
+        if s == 0 or not skip:
+            tin = step_inputs(w, s, w.ctx_len)
+            out = ec.ec_attend(d, to_dev(tin["q"]), to_dev(tin["k_new"]), to_dev(tin["v_new"]), gk, gv, None, dev_status=status)
+            want = oracle.refresh_and_attend(tin["q"], tin["k_new"], tin["v_new"], okc, ovc, None, w.dtype)
+            got = to_f64(out)
+        else:
+            n_partial += 1
+            assert st[3] == rows.size <= n_cap
+            assert idx_dev.cpu().numpy()[0, :rows.size].tolist() == rows.tolist()
+            tin = step_inputs(w, s, n_cap)     # the padded rows carry inputs too; their outputs are not used
+            out = ec.ec_attend(d, to_dev(tin["q"]), to_dev(tin["k_new"]), to_dev(tin["v_new"]), gk, gv, idx_dev, dev_status=status)
+            n = rows.size
+            want = oracle.refresh_and_attend(tin["q"][:, :n], tin["k_new"][:, :n], tin["v_new"][:, :n], okc, ovc,
+                                             rows[None, :].astype(np.int32), w.dtype)
+            got = to_f64(out)[:, :n]
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        err = np.abs(want - got).max()
+        assert err <= (1e-2 if w.dtype == syn.BF16 else 1e-5 * np.abs(want).max()), (s, err)
+        flags = decoded_this_step(host, s, 4)
+        if not flags.any():
+            host.masked[:] = True
+            flags = decoded_this_step(host, s, 4)
+        host.record(flags, 0)
+        o = oracle.entropy_gate(tin["logits"], w.dtype, w.vocab, flags, tau, w.block)
+        flags_dev = to_dev(flags)
+        g = ec.ec_entropy_gate(to_dev(tin["logits"]), w.vocab, w.block, flags_dev, tau)
+        assert abs(float(g["max_entropy"][0]) - o["max_entropy"][0]) <= 1e-4
+        assert abs(o["max_entropy"][0] - tau) >= 1e-4          # tau is a quantile of other steps' values or far away
+        assert int(g["decision"][0]) == int(o["decision"][0])
+        ec.ec_select_recent(hist, state, flags_dev, w0_dev, w.block, g["decision"], k, idx_dev)
+        R, skip, dt, t = oracle.step_bookkeeping(H, t, dt, w0 + np.flatnonzero(flags), int(o["decision"][0]), k)
+        rows = oracle.partial_step_rows(w0, w.block, R)
+        want_h = np.where(np.isfinite(H), H, -(2 ** 31)).astype(np.int64)
+        assert np.array_equal(hist.cpu().numpy()[0].astype(np.int64), want_h)
+    assert n_partial >= 2
+    assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)
