@@ -45,8 +45,8 @@ DEFAULT_WORKLOAD = "c2_llada_l768"
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
     "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-                    "sha256": "bb56071265acf609b4de4ef099da6642e6a7bdacb777b76370e8e1f4dca5bb13",
-                    "bytes_per_launch": {"c2_llada_l768": 12959744, "c5_llada_l4096": 68264192}},
+                    "sha256": "67630f6ddfc00b24fc9a8d18dbd9a73fbdcddf9dc0826592d3327fa6a0c71360",
+                    "bytes_per_launch": {"c2_llada_l768": 12965632, "c5_llada_l4096": 68294400}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
                      "sha256": "5904bb11f13265705d4e4f6ec7dd6af483762e10fe0d7d597d0c44524eb63616",
                      "bytes_per_launch": {"c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
