@@ -194,3 +194,47 @@ def partial_step_rows(window_start: int, block: int, R: np.ndarray) -> np.ndarra
     R = np.asarray(R, dtype=np.int64)
     outside = R[(R < window_start) | (R >= window_start + block)]
     return np.concatenate([window, np.sort(outside)])
+
+
+# --------------------------------------------------------------------------- #
+# Confidence-based parallel decoding behind the gate (Section 2.1; Section 5.1: threshold 0.9).
+# --------------------------------------------------------------------------- #
+def decode_confident(conf: np.ndarray, masked: np.ndarray, threshold: float) -> np.ndarray:
+    """Which rows of one sequence get decoded in this step: every still-masked row whose confidence (the
+    probability of its most likely token) exceeds `threshold`; when no masked row does, the masked row of the
+    highest confidence alone (the smallest index on ties), so that a step decodes at least one token while any is
+    masked.  The comparison is made on float32 values, the precision in which the confidences are produced and
+    the threshold is given.  Returns uint8 flags."""
+    c = np.asarray(conf, dtype=np.float64).astype(np.float32)
+    m = np.asarray(masked).astype(bool)
+    flags = m & (c > np.float32(threshold))
+    if not flags.any() and m.any():
+        cand = np.flatnonzero(m)
+        flags[cand[np.argmax(c[cand])]] = True          # argmax returns the first maximum: smallest index on ties
+    return flags.astype(np.uint8)
+
+
+def entropy_gate_decode(logits: np.ndarray, dtype: int, vocab: int, masked: np.ndarray, conf_threshold: float,
+                        tau: float, rows_per_seq: int) -> dict:
+    """Eq. 1 with the set D of newly decoded rows produced by the step itself: per-row statistics as in
+    entropy_gate, D from decode_confident per sequence, then E = max entropy over D and the comparison with tau.
+    Returns the statistics, `decoded` (uint8 per row), `masked_next` (masked minus decoded), `tokens` (argmax of
+    the decoded rows, -1 elsewhere), `max_entropy` and `decision` per sequence."""
+    masked = np.asarray(masked).astype(np.uint8)
+    stats = entropy_gate(logits, dtype, vocab, np.zeros(masked.size, np.uint8), tau, rows_per_seq)
+    decoded = np.zeros(masked.size, np.uint8)
+    for s0 in range(0, masked.size, rows_per_seq):
+        sl = slice(s0, s0 + rows_per_seq)
+        decoded[sl] = decode_confident(stats["conf"][sl], masked[sl], conf_threshold)
+    n_seq = masked.size // rows_per_seq
+    max_h = np.full(n_seq, -np.inf)
+    for b in range(n_seq):
+        sl = slice(b * rows_per_seq, (b + 1) * rows_per_seq)
+        h = stats["entropy"][sl][decoded[sl] != 0]
+        if h.size:
+            max_h[b] = h.max()
+    decision = (max_h > float(np.float32(tau))).astype(np.int32)
+    tokens = np.where(decoded != 0, stats["argmax"], -1).astype(np.int64)
+    return dict(argmax=stats["argmax"], conf=stats["conf"], entropy=stats["entropy"], decoded=decoded,
+                masked_next=(masked & (1 - decoded)).astype(np.uint8), tokens=tokens, max_entropy=max_h,
+                decision=decision)

@@ -490,3 +490,57 @@ def test_step_bookkeeping_follows_appendix_a_order():
     assert R.tolist() == [6, 7] and not skip and dt == 0 and t == 4
     rows = oracle.partial_step_rows(4, 4, np.array([1, 5, 9, 6]))
     assert rows.tolist() == [4, 5, 6, 7, 1, 9]
+
+
+# --------------------------------------------------------------------------- #
+# Confidence-based parallel decoding behind the gate (Section 2.1; threshold 0.9 in Section 5.1)
+# --------------------------------------------------------------------------- #
+def test_confident_rows_are_decoded_and_otherwise_the_single_best_masked_row():
+    f = lambda c, m, thr=0.9: oracle.decode_confident(np.array(c), np.array(m), thr).tolist()
+    assert f([0.95, 0.5, 0.91, 0.99], [1, 1, 0, 1]) == [1, 0, 0, 1]          # row 2 is confident but not masked
+    assert f([0.3, 0.8, 0.85, 0.85], [1, 0, 1, 1]) == [0, 0, 1, 0]           # nobody above 0.9: best masked row, first of the tie
+    assert f([0.3, 0.95, 0.2, 0.1], [1, 0, 1, 1]) == [1, 0, 0, 0]            # the confident row is unmasked: fallback among the masked
+    assert f([0.5, 0.6], [0, 0]) == [0, 0]                                   # nothing left to decode
+    assert f([np.float32(0.9), 0.2], [1, 1]) == [1, 0]                       # exactly the threshold is not above it: chosen only as the best
+    assert f([np.float32(0.9), np.nextafter(np.float32(0.9), np.float32(1))], [1, 1]) == [0, 1]
+    assert f([0.2, 0.4, 0.3], [1, 1, 1], thr=0.25) == [0, 1, 1]
+
+
+def test_gate_with_its_own_decoded_set_on_spike_and_flat_rows():
+    """Rows with one logit c above V - 1 zeros: conf = e^c / Z, H = ln Z - c e^c / Z, Z = e^c + V - 1 (closed form)."""
+    V = 16
+    cs = [10.0, 0.0, 6.0, 10.0, 2.0, 0.0]
+    lg = np.zeros((6, V), np.float32)
+    for r, c in enumerate(cs):
+        lg[r, (3 * r) % V] = c
+    Z = [math.exp(c) + V - 1 for c in cs]
+    conf = [math.exp(c) / z for c, z in zip(cs, Z)]
+    H = [math.log(z) - c * math.exp(c) / z for c, z in zip(cs, Z)]
+    assert conf[0] > 0.9 and conf[2] > 0.9 and conf[4] < 0.9
+    masked = np.array([1, 1, 1, 0, 1, 1], np.uint8)                           # row 3 was decoded earlier
+    o = oracle.entropy_gate_decode(lg, oracle.F32, V, masked, 0.9, tau=0.02, rows_per_seq=6)
+    assert o["decoded"].tolist() == [1, 0, 1, 0, 0, 0]
+    assert o["masked_next"].tolist() == [0, 1, 0, 0, 1, 1]
+    assert o["tokens"].tolist() == [0, -1, 6, -1, -1, -1]
+    assert abs(o["max_entropy"][0] - max(H[0], H[2])) < 1e-12 and o["max_entropy"][0] == pytest.approx(H[2])
+    assert o["decision"].tolist() == [1 if H[2] > 0.02 else 0]
+    # two sequences of three rows: the second has no confident masked row -> its best masked row (row 4) alone
+    o = oracle.entropy_gate_decode(lg, oracle.F32, V, np.array([1, 1, 1, 0, 1, 1], np.uint8), 0.9, tau=3.0, rows_per_seq=3)
+    assert o["decoded"].tolist() == [1, 0, 1, 0, 1, 0]
+    assert o["max_entropy"][1] == pytest.approx(H[4]) and o["decision"].tolist() == [0, 0]
+
+
+def test_decode_invariants_on_random_rows():
+    rng = np.random.Generator(np.random.PCG64(77))
+    for trial in range(50):
+        n = int(rng.integers(1, 40))
+        conf = rng.random(n) ** 0.3
+        masked = (rng.random(n) < 0.6).astype(np.uint8)
+        d = oracle.decode_confident(conf, masked, 0.9)
+        assert np.all(d <= masked)                                            # only masked rows are decoded
+        assert d.any() == masked.any()                                        # a step decodes something while anything is masked
+        above = (masked == 1) & (conf.astype(np.float32) > np.float32(0.9))
+        if above.any():
+            assert np.array_equal(d.astype(bool), above)
+        else:
+            assert d.sum() == int(masked.any())
