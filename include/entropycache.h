@@ -136,6 +136,29 @@ ec_status ec_entropy_gate(const void *logits, int32_t dtype, int32_t n_rows, int
                           float *max_entropy_out, int32_t *decision_out,
                           void *workspace, size_t workspace_bytes, void *stream);
 
+/* Largest rows_per_seq ec_entropy_gate_decode accepts. */
+#define EC_GATE_DECODE_MAX_ROWS_PER_SEQ 64
+
+/* The gate with confidence-based parallel decoding in front of it (Section 2.1 of the paper; its experiments use
+ * the threshold 0.9): the set D of newly decoded rows, which ec_entropy_gate takes as input, is formed inside the
+ * launch from the rows' confidences.  Per sequence b, with conf and argmax as ec_entropy_gate defines them:
+ *     decoded[r] = masked[r] != 0 && conf[r] > conf_threshold               (fp32 comparison)
+ *     if no row of the sequence qualifies and some row is masked: decoded[r*] = 1 for the masked row r* of the
+ *     highest confidence, the smallest index on ties (a step decodes at least one token while any is masked)
+ *     tokens[r] = argmax[r] and masked[r] = 0 for the decoded rows (other entries untouched)
+ *     decoded_flags_out[r] = decoded[r]   (the array ec_select_recent takes)
+ *     max_entropy_out[b] = max entropy over the decoded rows (-inf if none); decision_out[b] as ec_entropy_gate.
+ * masked: uint8 [n_rows], in/out; decoded_flags_out: uint8 [n_rows]; tokens: int32 [n_rows], in/out.
+ * rows_per_seq > EC_GATE_DECODE_MAX_ROWS_PER_SEQ returns EC_ERR_UNSUPPORTED.  Everything else (logits, optional
+ * row outputs, workspace, errors) as for ec_entropy_gate. */
+ec_status ec_entropy_gate_decode(const void *logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                                 int64_t row_stride_elems, int32_t rows_per_seq,
+                                 uint8_t *masked, float conf_threshold, float tau,
+                                 uint8_t *decoded_flags_out, int32_t *tokens,
+                                 int32_t *argmax_out, float *conf_out, float *entropy_out,
+                                 float *max_entropy_out, int32_t *decision_out,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+
 /* Largest n_rows ec_entropy_gate_static accepts. */
 #define EC_GATE_STATIC_MAX_ROWS 256
 

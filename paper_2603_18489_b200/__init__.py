@@ -62,6 +62,9 @@ def _load() -> ctypes.CDLL:
     lib.ec_entropy_gate.restype = i32
     lib.ec_entropy_gate_static.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
     lib.ec_entropy_gate_static.restype = i32
+    lib.ec_entropy_gate_decode.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, ctypes.c_float, vp, vp,
+                                           vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.ec_entropy_gate_decode.restype = i32
     lib.ec_select_recent.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, i32, vp, i32, vp]
     lib.ec_select_recent.restype = i32
     lib.ec_workspace_init.argtypes = [vp, sz, vp]
@@ -255,3 +258,39 @@ def ec_select_recent(history, state, decoded_flags, window_start, block: int, de
                                 _dev(decoded_flags, "decoded_flags"), _dev(window_start, "window_start"), int(block),
                                 _dev(decision, "decision"), int(k), _dev(active_idx, "active_idx"),
                                 int(active_idx.shape[1]), _stream(stream)), "ec_select_recent")
+
+
+def ec_entropy_gate_decode(logits, vocab: int, rows_per_seq: int, masked, conf_threshold: float, tau: float, tokens, *,
+                           decoded_out=None, argmax_out=None, conf_out=None, entropy_out=None, max_entropy_out=None,
+                           decision_out=None, workspace=None, want_rows: bool = True, stream=None) -> dict:
+    """The gate with confidence-based parallel decoding in front of it (argument marshalling only).  `masked`
+    (uint8 [R]) and `tokens` (int32 [R]) are updated in place.  Outputs are device tensors; nothing is synchronised."""
+    if logits.dim() != 2:
+        raise ValueError("logits must be [n_rows, row_stride]")
+    n_rows, stride = logits.shape
+    dev = logits.device
+    n_seq = n_rows // rows_per_seq if rows_per_seq > 0 else 0
+    if masked.dtype != torch.uint8 or tokens.dtype != torch.int32 or masked.numel() != n_rows or tokens.numel() != n_rows:
+        raise ValueError("masked must be uint8 [n_rows], tokens int32 [n_rows]")
+    if decoded_out is None:
+        decoded_out = torch.empty(n_rows, dtype=torch.uint8, device=dev)
+    if want_rows:
+        argmax_out = torch.empty(n_rows, dtype=torch.int32, device=dev) if argmax_out is None else argmax_out
+        conf_out = torch.empty(n_rows, dtype=torch.float32, device=dev) if conf_out is None else conf_out
+        entropy_out = torch.empty(n_rows, dtype=torch.float32, device=dev) if entropy_out is None else entropy_out
+    if max_entropy_out is None:
+        max_entropy_out = torch.empty(n_seq, dtype=torch.float32, device=dev)
+    if decision_out is None:
+        decision_out = torch.empty(n_seq, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = new_workspace(ec_entropy_gate_workspace_bytes(n_rows, vocab), dev)
+    _check(lib.ec_entropy_gate_decode(_dev(logits, "logits"), _dtype_code(logits), int(n_rows), int(vocab), int(stride),
+                                      int(rows_per_seq), _dev(masked, "masked"), float(conf_threshold), float(tau),
+                                      _dev(decoded_out, "decoded_out"), _dev(tokens, "tokens"),
+                                      _dev(argmax_out, "argmax_out"), _dev(conf_out, "conf_out"),
+                                      _dev(entropy_out, "entropy_out"), _dev(max_entropy_out, "max_entropy_out"),
+                                      _dev(decision_out, "decision_out"), _dev(workspace, "workspace"),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)),
+           "ec_entropy_gate_decode")
+    return dict(argmax=argmax_out, conf=conf_out, entropy=entropy_out, decoded=decoded_out, max_entropy=max_entropy_out,
+                decision=decision_out)

@@ -46,7 +46,13 @@ struct GateArgs {
     float* max_entropy_out;
     int* decision_out;
     void* workspace;
+    // decode mode (ec_entropy_gate_decode): the decoded set is formed inside the launch from the confidences
+    uint8_t* masked = nullptr;        // in/out, nullptr: the decoded set is `flags`
+    float conf_threshold = 0.f;
+    uint8_t* decoded_out = nullptr;
+    int* tokens = nullptr;
 };
+constexpr int kGateDecodeMaxRowsPerSeq = 64;
 size_t gate_workspace_bytes(int n_rows, int vocab);
 cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream);
 int select_recent_max_ctx();

@@ -183,6 +183,11 @@ struct GateParams {
     int* row_ticket;  // [n_rows], zero on entry, zero on exit
     int* seq_ticket;  // [n_seq],  zero on entry, zero on exit
     Partial* partials;  // [n_rows, splits]
+    // decode mode (masked != nullptr, single_level only): the decoded set comes from the confidences
+    uint8_t* masked;       // in/out [n_rows]: rows still masked; cleared for the rows decoded here
+    float conf_thr;
+    uint8_t* decoded_out;  // [n_rows]
+    int* tokens;           // [n_rows]: argmax written for the decoded rows
 };
 
 // warp-collective: merge the split partials of one row, write the row's outputs, return its entropy (all lanes)
@@ -220,6 +225,8 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     __shared__ int s_i[kGateThreads / 32];
     __shared__ float s_S[kGateThreads / 32], s_T[kGateThreads / 32];
     __shared__ float s_H[kSingleLevelMaxRows];
+    __shared__ float s_conf[kSingleLevelMaxRows];
+    __shared__ int s_arg[kSingleLevelMaxRows];
     __shared__ int s_last;
 
     constexpr int EPV = Loader<T>::EPV;
@@ -468,11 +475,62 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                 if (p.argmax_out) p.argmax_out[rr] = acc.idx;
                 if (p.conf_out) p.conf_out[rr] = conf;
                 p.entropy_out[rr] = H;
-                s_H[r] = p.flags[rr] ? H : -INFINITY;
+                if (p.masked) {
+                    s_H[r] = H;
+                    s_conf[r] = conf;
+                    s_arg[r] = acc.idx;
+                } else {
+                    s_H[r] = p.flags[rr] ? H : -INFINITY;
+                }
             }
         }
         __syncthreads();
-        if (warp == 0) {
+        if (warp == 0 && p.masked) {
+            // ---- confidence-based parallel decoding (Section 2.1 of the paper; threshold 0.9 in its experiments):
+            // every masked row above the threshold is decoded; if none is, the masked row of highest confidence
+            // (smallest index on ties).  Lane l owns rows l and l + 32 (rows_per_seq <= 64).
+            bool msk[2], dec[2];
+            float best = -1.f;
+            int best_r = 0x7fffffff;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int r = lane + 32 * q;
+                msk[q] = r < p.rows_per_seq && p.masked[seq * p.rows_per_seq + r] != 0;
+                dec[q] = msk[q] && s_conf[r] > p.conf_thr;
+                if (msk[q] && s_conf[r] > best) { best = s_conf[r]; best_r = r; }   // rows ascend: the first maximum stays
+            }
+            if (!__any_sync(0xffffffffu, dec[0] || dec[1])) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+                    const int orow = __shfl_xor_sync(0xffffffffu, best_r, o);
+                    if (ob > best || (ob == best && orow < best_r)) { best = ob; best_r = orow; }
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q) dec[q] = msk[q] && (lane + 32 * q == best_r);
+            }
+            float E = -INFINITY;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int r = lane + 32 * q;
+                if (r < p.rows_per_seq) {
+                    const int rr = seq * p.rows_per_seq + r;
+                    p.decoded_out[rr] = dec[q] ? 1 : 0;
+                    if (dec[q]) {
+                        p.tokens[rr] = s_arg[r];
+                        p.masked[rr] = 0;
+                        E = fmaxf(E, s_H[r]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+            if (lane == 0) {
+                p.max_entropy_out[seq] = E;
+                p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
+                p.seq_ticket[seq] = 0;   // ready for the next call
+            }
+        } else if (warp == 0) {
             float E = -INFINITY;
             for (int r = lane; r < p.rows_per_seq; r += 32) E = fmaxf(E, s_H[r]);
 #pragma unroll
@@ -527,12 +585,12 @@ GateWs carve(int n_rows) {
 
 // split count and columns per CTA: about one resident wave (4 CTAs of 256 threads per SM), every CTA a whole number
 // of 2048-column slabs, at most kMaxSplits partials per row
-void plan_chunks(int n_rows, int vocab, int* splits, int* chunk) {
+void plan_chunks(int n_rows, int vocab, int* splits, int* chunk, int max_splits = kMaxSplits) {
     const int slab = kGateThreads * kVec;
     const long long slots = 4LL * sm_count();
     long long want = slots / n_rows;
     if (want < 1) want = 1;
-    if (want > kMaxSplits) want = kMaxSplits;
+    if (want > max_splits) want = max_splits;
     long long per = (vocab + want - 1) / want;
     const long long per_min = (vocab + kMaxSplits - 1) / kMaxSplits;
     if (per < per_min) per = per_min;
@@ -585,9 +643,15 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     p.row_ticket = reinterpret_cast<int*>(ws + w.off_row);
     p.seq_ticket = reinterpret_cast<int*>(ws + w.off_seq);
     p.partials = reinterpret_cast<Partial*>(ws + w.off_part);
-    plan_chunks(a.n_rows, a.vocab, &p.splits, &p.chunk);
+    p.masked = a.masked;
+    p.conf_thr = a.conf_threshold;
+    p.decoded_out = a.decoded_out;
+    p.tokens = a.tokens;
+    // decode mode needs all rows of a sequence in one CTA's hands at the end: the single-level finish (at most 32 splits)
+    plan_chunks(a.n_rows, a.vocab, &p.splits, &p.chunk, a.masked ? 32 : kMaxSplits);
     if (p.splits > kMaxSplits) return cudaErrorInvalidValue;   // vocab > 96 * 8192: rejected by the API layer before this
     p.single_level = (a.rows_per_seq <= kSingleLevelMaxRows && p.splits <= 32) ? 1 : 0;
+    if (a.masked && !p.single_level) return cudaErrorInvalidValue;   // rows_per_seq > 64 or vocab > 32 * 8192 * ...: rejected by the API layer
     return a.dtype == EC_BF16 ? launch_t<__nv_bfloat16>(p, stream) : launch_t<float>(p, stream);
 }
 
