@@ -260,6 +260,17 @@ def _graph_time(torch, body, replays: int, warmup: int, stream) -> float:
     return e0.elapsed_time(e1) / replays
 
 
+def _workload(args) -> syn.Workload:
+    """The named workload, with the recent-token budget replaced when --k-recent is given (the paper's default is
+    k = 64 and its grid 16..256; BASELINE's configurations use 1..8)."""
+    import dataclasses
+
+    w = syn.WORKLOADS[args.workload]
+    if getattr(args, "k_recent", -1) >= 0:
+        w = dataclasses.replace(w, k_recent=args.k_recent)
+    return w
+
+
 def _choose_layers(w: syn.Workload) -> int:
     per_layer = 2 * w.batch * w.ctx_len * w.n_kv_heads * w.head_dim * syn.elem_bytes(w.dtype)
     need = int(np.ceil(3.0 * L2_BYTES / per_layer))
@@ -294,7 +305,7 @@ def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = syn.WORKLOADS[args.workload]
+    w = _workload(args)
     n_layers = _choose_layers(w)
     for _ in range(args.warmup):
         _oracle_layer_step_us(w, 1)
@@ -340,7 +351,7 @@ def run_cuda(args) -> None:
         dist = dist_
         dist.init_process_group("nccl", device_id=dev)
 
-    w = syn.WORKLOADS[args.workload]
+    w = _workload(args)
     n_layers = args.layers or _choose_layers(w)
     peaks = _peaks()
     if args.trace:
@@ -686,6 +697,8 @@ def main() -> None:
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--trace", action="store_true",
                     help="full-depth step trace of the workload (its layers and steps; decisions from the gate)")
+    ap.add_argument("--k-recent", type=int, default=-1,
+                    help="recent-token budget k of the skip step (rows = block + k); default: the workload's own")
     ap.add_argument("--only", default="", choices=["", "skip", "recompute", "gate"],
                     help="profiling aid: run only this part of the step")
     args = ap.parse_args()

@@ -48,7 +48,8 @@ constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr uint32_t STAGE = 2 * TILE;       // K tile + V tile: 64 KB
 constexpr uint32_t P_BYTES = SUB;          // P^T [128 keys x 64 query slots] bf16
 constexpr int kMaxStages = 3;
-constexpr int kMaxRowsT = 64;
+constexpr int kMaxRowsT = 64;            // query slots (packed rows) of one CTA
+constexpr int kMaxActive = 256;          // active rows of a sequence (refresh list, row chunks)
 constexpr uint32_t TM_COLS = 256;          // S^T buffers at columns 0 and 64, O^T at 128
 constexpr uint32_t TM_S = 0, TM_O = 128;
 // exchange areas, reusing the dead staging memory after the main loop (bytes from the aligned base)
@@ -104,8 +105,9 @@ struct KeysParams {
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads;
     int group;        // query heads of one kv head handled by one CTA column (a divisor of H_q / H_kv)
-    int n_sub;        // CTA columns per kv head = (H_q / H_kv) / group
-    int rows_total;   // n_active * group: packed query rows of one CTA
+    int rows_chunk;   // active rows handled by one CTA column (the last chunk may hold fewer)
+    int n_sub_r;      // row chunks = ceil(n_active / rows_chunk)
+    int n_sub;        // CTA columns per kv head = ((H_q / H_kv) / group) * n_sub_r
     int n_splits, tiles_per_split, n_stages;
     int q_tma;                    // 1: the producer fetches Q with one TMA box (MHA); 0: the softmax warps stage it
     uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0
@@ -142,7 +144,9 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int split = blockIdx.x, bh = blockIdx.y / p.n_sub, sub = blockIdx.y % p.n_sub;
     const int b = bh / p.n_kv_heads, hk = bh % p.n_kv_heads;
-    const int hq0 = (hk * p.n_sub + sub) * p.group;        // first query head of this CTA
+    const int hq0 = (hk * (p.n_sub / p.n_sub_r) + sub / p.n_sub_r) * p.group;   // first query head of this CTA
+    const int i0 = (sub % p.n_sub_r) * p.rows_chunk;                           // first active row of this CTA
+    const int rows_total = min(p.rows_chunk, p.n_active - i0) * p.group;       // packed query rows of this CTA
     const int C = p.n_splits;
     const int DL = HD / C;                                 // output columns this CTA merges
     const int n_tiles_total = (p.ctx_len + BK - 1) / BK;
@@ -200,7 +204,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (lane == 0) {
             if (p.q_tma) {   // Q first: [half][row][64 columns] of this head's rows, rows past n_active read as zero
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
-                tma_load_5d(base, &map_q, 0, 0, hq0, 0, b, bar(B_QFULL));
+                tma_load_5d(base, &map_q, 0, i0, hq0, 0, b, bar(B_QFULL));   // rows past the chunk land in unused slots
             }
             auto load_tile = [&](int tile, int stage) {
                 const int key0 = (t_begin + tile) * BK;
@@ -247,16 +251,16 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         // ================= refresh list, then MMA issue (lane 0) =================================
         bool spec_ok_w1 = true;
         if (refresh) {
-            int posv[kMaxRowsT / 32];
+            int posv[kMaxActive / 32];
 #pragma unroll
-            for (int k = 0; k < kMaxRowsT / 32; ++k) {
+            for (int k = 0; k < kMaxActive / 32; ++k) {
                 const int i = k * 32 + lane;
                 posv[k] = -1;
                 if (i < p.n_active) posv[k] = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
             }
             int n_mine = 0, hi_tile = -1, lo_tile = T;   // last / first local tile that holds a refreshed position
 #pragma unroll
-            for (int k = 0; k < kMaxRowsT / 32; ++k) {
+            for (int k = 0; k < kMaxActive / 32; ++k) {
                 const bool hit = posv[k] >= key_lo && posv[k] < key_hi;
                 const unsigned mk = __ballot_sync(0xffffffffu, hit);
                 if (hit) {
@@ -273,7 +277,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             if (n_mine > 0) rot = spec_ok_w1 ? hi_tile % (T - 1) : (hi_tile + 1) % T;   // (spec_ok and n_mine > 0 imply T > 1)
             int j_ref = T;
 #pragma unroll
-            for (int k = 0; k < kMaxRowsT / 32; ++k) {
+            for (int k = 0; k < kMaxActive / 32; ++k) {
                 if (posv[k] >= key_lo && posv[k] < key_hi) {
                     const int tile = (posv[k] - key_lo) / BK;
                     int j;
@@ -348,8 +352,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         for (int c = stid; c < (p.q_tma ? 0 : N * (HD / 8)); c += kSoft) {
             const int row = c >> 4, ch = c & 15;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (row < p.rows_total) {
-                const int i = row / p.group, jh = row % p.group;
+            if (row < rows_total) {
+                const int i = i0 + row / p.group, jh = row % p.group;
                 v = __ldg(reinterpret_cast<const uint4*>(
                     p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + ch * 8));
             }
@@ -535,8 +539,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             // ---- single CTA per (sequence, kv head): normalise and store column kk of every query row ----
 #pragma unroll
             for (int c = 0; c < N; ++c) {
-                if (c < p.rows_total) {
-                    const int i = c / p.group, jh = c % p.group;
+                if (c < rows_total) {
+                    const int i = i0 + c / p.group, jh = c % p.group;
                     __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD;
                     dst[kk] = __float2bfloat16_rn(__uint_as_float(o[c]) / sh->factor[c]);
                 }
@@ -585,14 +589,14 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             for (int s = 0; s < C; ++s) l = fmaf(fast_exp2(recv[s * cf + DL * NP + tid] - m), recv[s * cf + DL * NP + N + tid], l);
             const float inv = 1.f / l;
             for (int s = 0; s < C; ++s) wgt[s * N + tid] = fast_exp2(recv[s * cf + DL * NP + tid] - m) * inv;
-            const int i = tid / p.group, jh = tid % p.group;
+            const int i = i0 + tid / p.group, jh = tid % p.group;
             qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL;
         }
         __syncthreads();
         // a thread owns two adjacent output columns of a query row: one 4-byte store
         const int half_dl = DL / 2;
         const int dp = tid % half_dl;
-        for (int qq = tid / half_dl; qq < p.rows_total; qq += kThreads / half_dl) {
+        for (int qq = tid / half_dl; qq < rows_total; qq += kThreads / half_dl) {
             float a0 = 0.f, a1 = 0.f;
             for (int s = 0; s < C; ++s) {
                 const float w = wgt[s * N + qq];
@@ -662,7 +666,7 @@ bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_
 }
 
 struct KeysPlan {
-    int group, n_sub;   // query heads per CTA column, CTA columns per kv head
+    int group, rows_chunk, n_sub_r, n_sub;   // heads and active rows per CTA column, row chunks, CTA columns per kv head
     int n_slots, n_splits, tiles_per_split, n_stages;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
 };
@@ -676,8 +680,13 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
     const int g = d.n_q_heads / d.n_kv_heads;
     pl.group = g;
     while (pl.group > 1 && (g % pl.group != 0 || (long long)n_active * pl.group > kMaxRowsT)) --pl.group;
-    pl.n_sub = g / pl.group;
-    const int rows = n_active * pl.group;
+    // more active rows than slots (the paper's default budget k = 64 gives 96): the rows are cut into equal chunks,
+    // one CTA column each
+    pl.n_sub_r = (n_active * pl.group + kMaxRowsT - 1) / kMaxRowsT;
+    pl.rows_chunk = (n_active + pl.n_sub_r - 1) / pl.n_sub_r;
+    pl.n_sub_r = (n_active + pl.rows_chunk - 1) / pl.rows_chunk;
+    pl.n_sub = (g / pl.group) * pl.n_sub_r;
+    const int rows = pl.rows_chunk * pl.group;
     pl.n_slots = rows <= 48 ? 48 : 64;
     const int key_tiles = (d.ctx_len + BK - 1) / BK;
     const int bh = d.batch * d.n_kv_heads * pl.n_sub;
@@ -742,12 +751,14 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
 
 bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
-    if (n_active > kMaxRowsT) return false;
+    if (n_active > kMaxActive) return false;
     const KeysPlan pl = make_keys_plan(d, n_active);
     if ((long long)d.batch * d.n_kv_heads * pl.n_sub > 65535) return false;   // grid.y
     // the exchange areas (row-sum scratch, staging, receive buffer) reuse the memory below the refresh list
     // one CTA per SM: beyond one wave of CTAs the row-major skip kernel (two CTAs per SM) streams better
     if ((long long)pl.n_splits * d.batch * d.n_kv_heads * pl.n_sub > sm_count()) return false;
+    // row chunks re-read the K/V of a head once per chunk: only worth it while the keys can still be split
+    if (pl.n_sub_r > 1 && pl.n_splits < 2) return false;
     return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && kRecvOff + kExchangeMax <= pl.off_list;
 }
 
@@ -775,8 +786,9 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.n_q_heads = a.d.n_q_heads;
     p.n_kv_heads = a.d.n_kv_heads;
     p.group = pl.group;
+    p.rows_chunk = pl.rows_chunk;
+    p.n_sub_r = pl.n_sub_r;
     p.n_sub = pl.n_sub;
-    p.rows_total = a.n_active * p.group;
     p.n_splits = pl.n_splits;
     p.tiles_per_split = pl.tiles_per_split;
     p.n_stages = pl.n_stages;

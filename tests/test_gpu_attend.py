@@ -163,6 +163,19 @@ def test_grouped_query_skip_steps_spread_over_head_columns(Hq, Hkv, n, L):
     _check(w, t, refresh=False)
 
 
+@pytest.mark.parametrize("Hq,Hkv,n,L", [(32, 32, 96, 768), (8, 8, 70, 1000), (4, 4, 256, 640), (28, 4, 96, 768),
+                                        (6, 2, 129, 515), (16, 16, 160, 2048)])
+def test_skip_steps_with_more_active_rows_than_query_slots(Hq, Hkv, n, L):
+    """The paper's default budget k = 64 gives 96 active rows, its grid up to 288: the active rows are cut into
+    chunks of at most 64 packed rows, one CTA column each (48 + 48 at n = 96, 35 + 35 at n = 70, four chunks at
+    256, with GQA on top: 2 row chunks x 7 head columns), every column refreshing the whole list's rows."""
+    w = syn.Workload(96, "row_chunks", syn.BF16, 1, Hq, Hkv, 128, 0, L, 1, 0, 64)
+    idx = syn.arbitrary_active_idx(1, L, n, seed=13 * L + n)
+    t = syn.attn_inputs(w, n, active_idx=idx, std_qk=0.7, std_v=0.5)
+    _check(w, t)
+    _check(w, t, refresh=False)
+
+
 def test_few_row_skip_step_with_rising_maxima():
     """Keys ordered so that the row maxima keep rising from tile to tile (scores grow with the position): the
     lazily updated references must be raised, and the accumulator rescaled, several times."""
