@@ -51,8 +51,8 @@ NCU_TRAFFIC = {
                      "sha256": "5904bb11f13265705d4e4f6ec7dd6af483762e10fe0d7d597d0c44524eb63616",
                      "bytes_per_launch": {"c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
     "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
-                     "sha256": "f7350fa75a2ea8d82120fbfb3ea587e366e2a8716e4a2a11e71f8f323e1ef9f3",
-                     "bytes_per_launch": {"c5_llada_l4096_b8": 65324032}},
+                     "sha256": "08db22804ea2a9ba21796a5779146a48da833acacebe4fcd94b12ec2ec51e273",
+                     "bytes_per_launch": {"c5_llada_l4096_b8": 65467904}},
 }
 
 
