@@ -238,3 +238,25 @@ def entropy_gate_decode(logits: np.ndarray, dtype: int, vocab: int, masked: np.n
     return dict(argmax=stats["argmax"], conf=stats["conf"], entropy=stats["entropy"], decoded=decoded,
                 masked_next=(masked & (1 - decoded)).astype(np.uint8), tokens=tokens, max_entropy=max_h,
                 decision=decision)
+
+
+# --------------------------------------------------------------------------- #
+# The three candidate gate metrics of Section 5.3 ("Choice of Thresholding Variable").
+# --------------------------------------------------------------------------- #
+def gate_metrics(entropy: np.ndarray, conf: np.ndarray, decoded_flags: np.ndarray, rows_per_seq: int) -> dict:
+    """Per sequence, over its newly decoded rows D: (1) max entropy = max_{i in D} e(p_i), the metric of Eq. 1;
+    (2) entropy sum = sum_{i in D} e(p_i); (3) max confidence = max_{i in D} max_j p_ij.  An empty D gives -inf, 0
+    and -inf.  Inputs are the per-row entropies and confidences of entropy_gate."""
+    e = np.asarray(entropy, dtype=np.float64)
+    c = np.asarray(conf, dtype=np.float64)
+    f = np.asarray(decoded_flags).astype(bool)
+    n_seq = e.size // rows_per_seq
+    out = dict(max_entropy=np.full(n_seq, -np.inf), entropy_sum=np.zeros(n_seq), max_conf=np.full(n_seq, -np.inf))
+    for b in range(n_seq):
+        sl = slice(b * rows_per_seq, (b + 1) * rows_per_seq)
+        d = f[sl]
+        if d.any():
+            out["max_entropy"][b] = e[sl][d].max()
+            out["entropy_sum"][b] = e[sl][d].sum()
+            out["max_conf"][b] = c[sl][d].max()
+    return out

@@ -544,3 +544,34 @@ def test_decode_invariants_on_random_rows():
             assert np.array_equal(d.astype(bool), above)
         else:
             assert d.sum() == int(masked.any())
+
+
+# --------------------------------------------------------------------------- #
+# The three candidate gate metrics (Section 5.3)
+# --------------------------------------------------------------------------- #
+def test_gate_metrics_on_hand_worked_rows():
+    ent = np.array([0.5, 2.0, 0.25, 1.0, 3.0, 0.125])
+    conf = np.array([0.9, 0.3, 0.95, 0.6, 0.1, 0.99])
+    flags = np.array([1, 0, 1, 1, 0, 0], np.uint8)
+    m = oracle.gate_metrics(ent, conf, flags, 6)
+    assert m["max_entropy"].tolist() == [1.0] and m["entropy_sum"].tolist() == [1.75] and m["max_conf"].tolist() == [0.95]
+    m = oracle.gate_metrics(ent, conf, flags, 3)                      # two sequences of three rows
+    assert m["max_entropy"].tolist() == [0.5, 1.0] and m["entropy_sum"].tolist() == [0.75, 1.0]
+    assert m["max_conf"].tolist() == [0.95, 0.6]
+    m = oracle.gate_metrics(ent, conf, np.zeros(6, np.uint8), 6)      # nothing decoded
+    assert np.isneginf(m["max_entropy"][0]) and m["entropy_sum"][0] == 0.0 and np.isneginf(m["max_conf"][0])
+
+
+def test_gate_metrics_agree_with_the_gate_and_with_each_other():
+    V, R = 300, 24
+    d = syn.logits_rows(R, V, syn.F32, cfg_id=88)
+    flags = syn.decoded_flags(R, 3, 8, cfg_id=88)
+    g = oracle.entropy_gate(d["logits"], syn.F32, V, flags, 1.0, 8)
+    m = oracle.gate_metrics(g["entropy"], g["conf"], flags, 8)
+    assert np.array_equal(m["max_entropy"], g["max_entropy"])        # metric (1) is Eq. 1's E
+    for b in range(3):
+        n = int(flags[8 * b:8 * b + 8].sum())
+        assert m["max_entropy"][b] <= m["entropy_sum"][b] + 1e-15 <= n * m["max_entropy"][b] + 1e-12
+        assert 1.0 / V <= m["max_conf"][b] <= 1.0
+        # the most confident decoded row has at most -ln(conf) ... entropy bound from below: H >= -ln(max p)
+        assert m["max_entropy"][b] >= -math.log(m["max_conf"][b]) - 1e-12 or n > 1
