@@ -136,6 +136,21 @@ ec_status ec_entropy_gate(const void *logits, int32_t dtype, int32_t n_rows, int
                           float *max_entropy_out, int32_t *decision_out,
                           void *workspace, size_t workspace_bytes, void *stream);
 
+/* ec_entropy_gate with the other two candidate metrics of Section 5.3 ("Choice of Thresholding Variable") as
+ * extra per-sequence outputs, over the same set D of decoded rows:
+ *     entropy_sum_out[b] = sum over D of entropy   (0 if D is empty)
+ *     max_conf_out[b]    = max over D of conf      (-inf if D is empty)
+ * decision_out still applies Eq. 1's rule to the maximum entropy; thresholding the other two is the caller's.
+ * Either extra pointer may be NULL.  rows_per_seq is limited to EC_GATE_DECODE_MAX_ROWS_PER_SEQ when one of them
+ * is given (EC_ERR_UNSUPPORTED beyond).  Everything else as for ec_entropy_gate. */
+ec_status ec_entropy_gate_metrics(const void *logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                                  int64_t row_stride_elems, int32_t rows_per_seq,
+                                  const uint8_t *decoded_flags, float tau,
+                                  int32_t *argmax_out, float *conf_out, float *entropy_out,
+                                  float *max_entropy_out, int32_t *decision_out,
+                                  float *entropy_sum_out, float *max_conf_out,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+
 /* Largest rows_per_seq ec_entropy_gate_decode accepts. */
 #define EC_GATE_DECODE_MAX_ROWS_PER_SEQ 64
 

@@ -62,6 +62,9 @@ def _load() -> ctypes.CDLL:
     lib.ec_entropy_gate.restype = i32
     lib.ec_entropy_gate_static.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
     lib.ec_entropy_gate_static.restype = i32
+    lib.ec_entropy_gate_metrics.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp,
+                                            vp, sz, vp]
+    lib.ec_entropy_gate_metrics.restype = i32
     lib.ec_entropy_gate_decode.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, ctypes.c_float, vp, vp,
                                            vp, vp, vp, vp, vp, vp, sz, vp]
     lib.ec_entropy_gate_decode.restype = i32
@@ -294,3 +297,29 @@ def ec_entropy_gate_decode(logits, vocab: int, rows_per_seq: int, masked, conf_t
            "ec_entropy_gate_decode")
     return dict(argmax=argmax_out, conf=conf_out, entropy=entropy_out, decoded=decoded_out, max_entropy=max_entropy_out,
                 decision=decision_out)
+
+
+def ec_entropy_gate_metrics(logits, vocab: int, rows_per_seq: int, decoded_flags, tau: float, *, workspace=None,
+                            stream=None) -> dict:
+    """ec_entropy_gate plus the entropy sum and the maximum confidence over the decoded rows (Section 5.3 of the
+    paper); argument marshalling only.  Outputs are device tensors; nothing is synchronised."""
+    if logits.dim() != 2:
+        raise ValueError("logits must be [n_rows, row_stride]")
+    n_rows, stride = logits.shape
+    dev = logits.device
+    n_seq = n_rows // rows_per_seq if rows_per_seq > 0 else 0
+    f32 = lambda n: torch.empty(n, dtype=torch.float32, device=dev)
+    out = dict(argmax=torch.empty(n_rows, dtype=torch.int32, device=dev), conf=f32(n_rows), entropy=f32(n_rows),
+               max_entropy=f32(n_seq), decision=torch.empty(n_seq, dtype=torch.int32, device=dev),
+               entropy_sum=f32(n_seq), max_conf=f32(n_seq))
+    if workspace is None:
+        workspace = new_workspace(ec_entropy_gate_workspace_bytes(n_rows, vocab), dev)
+    _check(lib.ec_entropy_gate_metrics(_dev(logits, "logits"), _dtype_code(logits), int(n_rows), int(vocab), int(stride),
+                                       int(rows_per_seq), _dev(decoded_flags, "decoded_flags"), float(tau),
+                                       _dev(out["argmax"], "argmax"), _dev(out["conf"], "conf"),
+                                       _dev(out["entropy"], "entropy"), _dev(out["max_entropy"], "max_entropy"),
+                                       _dev(out["decision"], "decision"), _dev(out["entropy_sum"], "entropy_sum"),
+                                       _dev(out["max_conf"], "max_conf"), _dev(workspace, "workspace"),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)),
+           "ec_entropy_gate_metrics")
+    return out

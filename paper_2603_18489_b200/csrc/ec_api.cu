@@ -176,8 +176,8 @@ namespace {
 ec_status gate_call(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride_elems,
                     int32_t rows_per_seq, const uint8_t* decoded_flags, uint8_t* masked, float conf_threshold,
                     uint8_t* decoded_out, int32_t* tokens, float tau, int32_t* argmax_out, float* conf_out,
-                    float* entropy_out, float* max_entropy_out, int32_t* decision_out, void* workspace,
-                    size_t workspace_bytes, void* stream) {
+                    float* entropy_out, float* max_entropy_out, int32_t* decision_out, float* entropy_sum_out,
+                    float* max_conf_out, void* workspace, size_t workspace_bytes, void* stream) {
     if (dtype != EC_F32 && dtype != EC_BF16) return EC_ERR_DTYPE;
     if (n_rows < 0 || vocab < 1 || rows_per_seq < 1 || row_stride_elems < vocab) return EC_ERR_SHAPE;
     if (n_rows % rows_per_seq != 0) return EC_ERR_SHAPE;
@@ -186,7 +186,8 @@ ec_status gate_call(const void* logits, int32_t dtype, int32_t n_rows, int32_t v
     if (tau != tau) return EC_ERR_SHAPE;
     const bool decode = masked != nullptr || decoded_out != nullptr || tokens != nullptr;
     if (decode && (conf_threshold != conf_threshold)) return EC_ERR_SHAPE;
-    if (decode && rows_per_seq > kGateDecodeMaxRowsPerSeq) return EC_ERR_UNSUPPORTED;
+    const bool one_cta_finish = decode || entropy_sum_out != nullptr || max_conf_out != nullptr;
+    if (one_cta_finish && rows_per_seq > kGateDecodeMaxRowsPerSeq) return EC_ERR_UNSUPPORTED;
     if (n_rows == 0) return EC_OK;
     if (!logits || !max_entropy_out || !decision_out) return EC_ERR_NULL;
     if (decode ? (!masked || !decoded_out || !tokens) : !decoded_flags) return EC_ERR_NULL;
@@ -194,7 +195,8 @@ ec_status gate_call(const void* logits, int32_t dtype, int32_t n_rows, int32_t v
     if (!aligned16(logits) || ((size_t)row_stride_elems * esize) % 16 != 0) return EC_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(argmax_out) | reinterpret_cast<uintptr_t>(conf_out) |
          reinterpret_cast<uintptr_t>(entropy_out) | reinterpret_cast<uintptr_t>(max_entropy_out) |
-         reinterpret_cast<uintptr_t>(decision_out) | reinterpret_cast<uintptr_t>(tokens)) & 3u)
+         reinterpret_cast<uintptr_t>(decision_out) | reinterpret_cast<uintptr_t>(tokens) |
+         reinterpret_cast<uintptr_t>(entropy_sum_out) | reinterpret_cast<uintptr_t>(max_conf_out)) & 3u)
         return EC_ERR_ALIGN;
     const size_t need = gate_workspace_bytes(n_rows, vocab);
     if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
@@ -217,6 +219,8 @@ ec_status gate_call(const void* logits, int32_t dtype, int32_t n_rows, int32_t v
     a.conf_threshold = conf_threshold;
     a.decoded_out = decoded_out;
     a.tokens = tokens;
+    a.entropy_sum_out = entropy_sum_out;
+    a.max_conf_out = max_conf_out;
     const cudaError_t e = launch_gate(a, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
@@ -228,8 +232,18 @@ ec_status ec_entropy_gate(const void* logits, int32_t dtype, int32_t n_rows, int
                           float* conf_out, float* entropy_out, float* max_entropy_out, int32_t* decision_out,
                           void* workspace, size_t workspace_bytes, void* stream) {
     return gate_call(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags, nullptr, 0.f, nullptr,
-                     nullptr, tau, argmax_out, conf_out, entropy_out, max_entropy_out, decision_out, workspace,
-                     workspace_bytes, stream);
+                     nullptr, tau, argmax_out, conf_out, entropy_out, max_entropy_out, decision_out, nullptr, nullptr,
+                     workspace, workspace_bytes, stream);
+}
+
+ec_status ec_entropy_gate_metrics(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                                  int64_t row_stride_elems, int32_t rows_per_seq, const uint8_t* decoded_flags, float tau,
+                                  int32_t* argmax_out, float* conf_out, float* entropy_out, float* max_entropy_out,
+                                  int32_t* decision_out, float* entropy_sum_out, float* max_conf_out, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+    return gate_call(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags, nullptr, 0.f, nullptr,
+                     nullptr, tau, argmax_out, conf_out, entropy_out, max_entropy_out, decision_out, entropy_sum_out,
+                     max_conf_out, workspace, workspace_bytes, stream);
 }
 
 ec_status ec_entropy_gate_decode(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
@@ -240,7 +254,7 @@ ec_status ec_entropy_gate_decode(const void* logits, int32_t dtype, int32_t n_ro
     if (!masked || !decoded_flags_out || !tokens) return n_rows == 0 ? EC_OK : EC_ERR_NULL;
     return gate_call(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, nullptr, masked, conf_threshold,
                      decoded_flags_out, tokens, tau, argmax_out, conf_out, entropy_out, max_entropy_out, decision_out,
-                     workspace, workspace_bytes, stream);
+                     nullptr, nullptr, workspace, workspace_bytes, stream);
 }
 
 ec_status ec_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

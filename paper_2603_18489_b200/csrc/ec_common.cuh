@@ -51,6 +51,9 @@ struct GateArgs {
     float conf_threshold = 0.f;
     uint8_t* decoded_out = nullptr;
     int* tokens = nullptr;
+    // the other two candidate metrics of Section 5.3 over the decoded rows (optional, per sequence)
+    float* entropy_sum_out = nullptr;
+    float* max_conf_out = nullptr;
 };
 constexpr int kGateDecodeMaxRowsPerSeq = 64;
 size_t gate_workspace_bytes(int n_rows, int vocab);

@@ -188,6 +188,9 @@ struct GateParams {
     float conf_thr;
     uint8_t* decoded_out;  // [n_rows]
     int* tokens;           // [n_rows]: argmax written for the decoded rows
+    // Section 5.3's other candidate metrics over the decoded rows (single_level only; either may be null)
+    float* ent_sum_out;    // [n_seq]
+    float* max_conf_out;   // [n_seq]
 };
 
 // warp-collective: merge the split partials of one row, write the row's outputs, return its entropy (all lanes)
@@ -481,6 +484,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                     s_arg[r] = acc.idx;
                 } else {
                     s_H[r] = p.flags[rr] ? H : -INFINITY;
+                    s_conf[r] = p.flags[rr] ? conf : -INFINITY;
                 }
             }
         }
@@ -509,7 +513,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
 #pragma unroll
                 for (int q = 0; q < 2; ++q) dec[q] = msk[q] && (lane + 32 * q == best_r);
             }
-            float E = -INFINITY;
+            float E = -INFINITY, Hsum = 0.f, Cmax = -INFINITY;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int r = lane + 32 * q;
@@ -520,22 +524,40 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                         p.tokens[rr] = s_arg[r];
                         p.masked[rr] = 0;
                         E = fmaxf(E, s_H[r]);
+                        Hsum += s_H[r];
+                        Cmax = fmaxf(Cmax, s_conf[r]);
                     }
                 }
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+            for (int o = 16; o > 0; o >>= 1) {
+                E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+                Hsum += __shfl_xor_sync(0xffffffffu, Hsum, o);
+                Cmax = fmaxf(Cmax, __shfl_xor_sync(0xffffffffu, Cmax, o));
+            }
             if (lane == 0) {
+                if (p.ent_sum_out) p.ent_sum_out[seq] = Hsum;
+                if (p.max_conf_out) p.max_conf_out[seq] = Cmax;
                 p.max_entropy_out[seq] = E;
                 p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
                 p.seq_ticket[seq] = 0;   // ready for the next call
             }
         } else if (warp == 0) {
-            float E = -INFINITY;
-            for (int r = lane; r < p.rows_per_seq; r += 32) E = fmaxf(E, s_H[r]);
+            float E = -INFINITY, Hsum = 0.f, Cmax = -INFINITY;
+            for (int r = lane; r < p.rows_per_seq; r += 32) {
+                E = fmaxf(E, s_H[r]);
+                Hsum += (s_H[r] == -INFINITY) ? 0.f : s_H[r];   // rows outside the decoded set carry -inf
+                Cmax = fmaxf(Cmax, s_conf[r]);
+            }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+            for (int o = 16; o > 0; o >>= 1) {
+                E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
+                Hsum += __shfl_xor_sync(0xffffffffu, Hsum, o);
+                Cmax = fmaxf(Cmax, __shfl_xor_sync(0xffffffffu, Cmax, o));
+            }
             if (lane == 0) {
+                if (p.ent_sum_out) p.ent_sum_out[seq] = Hsum;
+                if (p.max_conf_out) p.max_conf_out[seq] = Cmax;
                 p.max_entropy_out[seq] = E;
                 p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
                 p.seq_ticket[seq] = 0;   // ready for the next call
@@ -647,11 +669,15 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     p.conf_thr = a.conf_threshold;
     p.decoded_out = a.decoded_out;
     p.tokens = a.tokens;
-    // decode mode needs all rows of a sequence in one CTA's hands at the end: the single-level finish (at most 32 splits)
-    plan_chunks(a.n_rows, a.vocab, &p.splits, &p.chunk, a.masked ? 32 : kMaxSplits);
+    p.ent_sum_out = a.entropy_sum_out;
+    p.max_conf_out = a.max_conf_out;
+    // decode mode and the extra metrics need all rows of a sequence in one CTA's hands at the end: the single-level
+    // finish (at most 32 splits)
+    const bool one_cta_finish = a.masked || a.entropy_sum_out || a.max_conf_out;
+    plan_chunks(a.n_rows, a.vocab, &p.splits, &p.chunk, one_cta_finish ? 32 : kMaxSplits);
     if (p.splits > kMaxSplits) return cudaErrorInvalidValue;   // vocab > 96 * 8192: rejected by the API layer before this
     p.single_level = (a.rows_per_seq <= kSingleLevelMaxRows && p.splits <= 32) ? 1 : 0;
-    if (a.masked && !p.single_level) return cudaErrorInvalidValue;   // rows_per_seq > 64 or vocab > 32 * 8192 * ...: rejected by the API layer
+    if (one_cta_finish && !p.single_level) return cudaErrorInvalidValue;   // rows_per_seq > 64 or vocab > 32 * 8192 * ...: rejected by the API layer
     return a.dtype == EC_BF16 ? launch_t<__nv_bfloat16>(p, stream) : launch_t<float>(p, stream);
 }
 

@@ -132,3 +132,27 @@ def test_gate_shift_invariance_on_device():
     a = _run_gpu(d["logits"], syn.F32, w.vocab, flags, 1.5, 32)
     b = _run_gpu(d["logits"] + np.float32(16.0), syn.F32, w.vocab, flags, 1.5, 32)
     assert np.abs(a["entropy"] - b["entropy"]).max() < 5e-5
+
+
+@pytest.mark.parametrize("name,R,rps", [("c1_tiny_fp32", 32, 32), ("c2_llada_l768", 32, 32), ("c5_llada_l4096_b8", 256, 32),
+                                        ("c1_tiny_fp32", 15, 5), ("c3_dream_l768", 128, 64)])
+def test_the_three_candidate_metrics(name, R, rps):
+    """Section 5.3: max entropy, entropy sum and max confidence over the decoded rows, per sequence; empty decoded sets
+    included (one sequence gets no flags).  Sum: within 1e-4 nats per decoded row; confidence: 1e-5 relative."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.WORKLOADS[name]
+    d = syn.logits_rows(R, w.vocab, w.dtype, cfg_id=w.cfg_id, salt=3)
+    flags = syn.decoded_flags(R, max(1, rps // 3), rps, cfg_id=w.cfg_id)
+    flags[:rps] = 0                                                   # the first sequence decodes nothing
+    o = oracle.entropy_gate(d["logits"], w.dtype, w.vocab, flags, 1.5, rps)
+    m = oracle.gate_metrics(o["entropy"], o["conf"], flags, rps)
+    g = ec.ec_entropy_gate_metrics(to_dev(d["logits"]), w.vocab, rps, to_dev(flags), 1.5)
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in g.items()}
+    _compare(g, o, 1.5)
+    n_dec = flags.reshape(-1, rps).sum(axis=1)
+    assert np.all(np.abs(g["entropy_sum"].astype(np.float64) - m["entropy_sum"]) <= ENT_TOL * np.maximum(n_dec, 1))
+    fin = np.isfinite(m["max_conf"])
+    assert np.array_equal(np.isfinite(g["max_conf"]), fin) and not fin[0] and g["entropy_sum"][0] == 0.0
+    assert np.all(np.abs(g["max_conf"][fin].astype(np.float64) - m["max_conf"][fin]) <= 1e-5 * m["max_conf"][fin])
