@@ -118,3 +118,69 @@ def run_replay(w: syn.Workload, n_steps: int, tau: float, k: int, attend_fn, gat
                             used=int(used), idx=idx))
         st.record(flags, used)
     return records
+
+
+class SlidingState:
+    """Sliding-window decoding (Section 2.1 of the paper: the window advances over the sequence and keeps the number of
+    masked tokens being denoised constant): the window of a step is the first `window` still-masked positions of the
+    generation region, which stop being contiguous as soon as a position inside is decoded.  Same history / skip_flag /
+    dt bookkeeping as ReplayState."""
+
+    def __init__(self, w: syn.Workload, window: int):
+        self.w, self.window = w, window
+        self.t, self.dt, self.skip_flag = 0, 0, False
+        self.H = np.full(w.ctx_len, -np.inf)
+        self.masked = np.zeros(w.ctx_len, dtype=bool)
+        self.masked[w.prompt_len:] = True
+
+    def window_positions(self) -> np.ndarray:
+        return np.flatnonzero(self.masked)[:self.window].astype(np.int32)
+
+    def recent_rows(self, k: int) -> np.ndarray:
+        decoded = np.flatnonzero(np.isfinite(self.H))
+        if k == 0 or decoded.size == 0:
+            return np.empty(0, np.int32)
+        order = decoded[np.argsort(-self.H[decoded], kind="stable")]
+        tau_r = max(self.H[order[:k]].min(), self.t - self.dt)
+        return np.sort(decoded[self.H[decoded] >= tau_r]).astype(np.int32)
+
+    def active_rows(self, k: int) -> np.ndarray | None:
+        if self.t == 0 or not self.skip_flag:
+            return None
+        win = self.window_positions()
+        rec = self.recent_rows(k)
+        return np.concatenate([win, rec[~np.isin(rec, win)]]).astype(np.int32)
+
+    def record(self, decoded_pos: np.ndarray, decision: int) -> None:
+        self.H[decoded_pos] = self.t
+        self.masked[decoded_pos] = False
+        self.skip_flag = decision == 0
+        self.dt = self.dt + 1 if self.skip_flag else 0
+        self.t += 1
+
+
+def run_replay_sliding(w: syn.Workload, window: int, n_steps: int, tau: float, k: int, attend_fn, gate_fn,
+                       forced_decisions=None, per_step: int = 3):
+    """The sliding-window counterpart of run_replay: the gate sees the logits rows of the window's positions (one row
+    per window position, `window` rows per sequence), a seeded choice of them is decoded each step."""
+    st = SlidingState(w, window)
+    records = []
+    for s in range(n_steps):
+        win = st.window_positions()
+        if win.size < window:          # the generation region is nearly finished: stop the trace
+            break
+        idx = st.active_rows(k)
+        n_active = w.ctx_len if idx is None else idx.size
+        t = step_inputs(w, s, n_active)
+        idx_b = None if idx is None else np.broadcast_to(idx, (w.batch, n_active)).copy()
+        out = attend_fn(t["q"], t["k_new"], t["v_new"], idx_b)
+        rng = np.random.Generator(np.random.PCG64(4242 + 100000 * s + w.cfg_id))
+        flags = np.zeros(window, np.uint8)
+        flags[rng.choice(window, size=min(per_step, window), replace=False)] = 1
+        lg = syn.logits_rows(window, w.vocab, w.dtype, cfg_id=w.cfg_id, step=s)["logits"]
+        E, dec = gate_fn(lg, flags, tau)
+        used = dec if forced_decisions is None or forced_decisions[s] is None else forced_decisions[s]
+        records.append(dict(step=s, full=idx is None, n_active=n_active, out=out, E=float(E), decision=int(dec),
+                            used=int(used), idx=idx))
+        st.record(win[flags != 0], used)
+    return records

@@ -9,7 +9,7 @@ import torch
 
 import ec_synth as syn
 import oracle
-from _replay import run_replay, step_inputs, ReplayState, decoded_this_step
+from _replay import run_replay, run_replay_sliding, step_inputs, ReplayState, decoded_this_step
 from _util import to_dev, to_f64, to_storage
 
 pytestmark = pytest.mark.gpu
@@ -177,4 +177,45 @@ def test_loop_state_kept_on_the_device(name, k, n_steps):
         want_h = np.where(np.isfinite(H), H, -(2 ** 31)).astype(np.int64)
         assert np.array_equal(hist.cpu().numpy()[0].astype(np.int64), want_h)
     assert n_partial >= 2
+    assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)
+
+
+@pytest.mark.parametrize("name,window,k", [("c1_tiny_fp32", 8, 2), ("c2_llada_l768", 32, 4), ("c3_dream_l768", 32, 2),
+                                            ("c2_llada_l768", 64, 8), ("c4_llada_l2048", 128, 2)])
+def test_sliding_window_replay(name, window, k):
+    """Sliding-window decoding (the paper's evaluation mode, window 32; its appendix varies the window from 8 to 128):
+    the window is the first `window` still-masked positions, non-contiguous after the first decode, so the row lists
+    are arbitrary ascending sets plus the recent rows; LLaDA and Dream (GQA) geometries."""
+    w = syn.WORKLOADS[name]
+    n_steps = 10
+    kc, vc = _caches(w)
+    okc, ovc = kc.copy(), vc.copy()
+    o_att, _ = _oracle_fns(w, okc, ovc)
+
+    def o_gate(logits, flags, tau):
+        o = oracle.entropy_gate(logits, w.dtype, w.vocab, flags, tau, window)
+        return o["max_entropy"][0], int(o["decision"][0])
+
+    probe = run_replay_sliding(w, window, n_steps, 0.0, k, lambda *a: np.zeros(1), o_gate)
+    tau = float(np.float32(np.quantile([r["E"] for r in probe], 0.7)))     # about a third of the steps recompute
+    ref = run_replay_sliding(w, window, n_steps, tau, k, o_att, o_gate)
+    gk, gv = to_dev(kc), to_dev(vc)
+    g_att, _ = _gpu_fns(w, gk, gv)
+
+    def g_gate(logits, flags, tau):
+        import paper_2603_18489_b200 as ec
+
+        r = ec.ec_entropy_gate(to_dev(logits), w.vocab, window, to_dev(flags), tau)
+        torch.cuda.synchronize()
+        return float(r["max_entropy"][0]), int(r["decision"][0])
+
+    got = run_replay_sliding(w, window, n_steps, tau, k, g_att, g_gate, forced_decisions=[r["decision"] for r in ref])
+    assert len(ref) == len(got) >= 6 and any(not r["full"] for r in ref[1:])
+    for a, b in zip(ref, got):
+        assert a["full"] == b["full"] and a["n_active"] == b["n_active"]
+        err = np.abs(a["out"] - b["out"]).max()
+        assert err <= (1e-2 if w.dtype == syn.BF16 else 1e-5 * np.abs(a["out"]).max()), (a["step"], err)
+        assert abs(a["E"] - b["E"]) <= 1e-4
+        if abs(a["E"] - tau) >= 1e-4:
+            assert a["decision"] == b["decision"]
     assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)

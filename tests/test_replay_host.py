@@ -59,3 +59,18 @@ def test_replay_drives_both_branches_and_counts_dt():
     assert calls[0] is None                               # step 1 full
     assert [r["full"] for r in rec] == [True, False, False, True, False, True, True, False]
     assert all(c is None or c >= 32 for c in calls)
+
+
+def test_sliding_window_keeps_the_masked_count_constant_and_goes_non_contiguous():
+    from _replay import SlidingState
+
+    w = syn.C1
+    st = SlidingState(w, 8)
+    p0 = w.prompt_len
+    assert st.window_positions().tolist() == list(range(p0, p0 + 8))
+    st.record(np.array([p0 + 1, p0 + 4]), decision=0)
+    win = st.window_positions()
+    assert win.size == 8 and win.tolist() == [p0, p0 + 2, p0 + 3, p0 + 5, p0 + 6, p0 + 7, p0 + 8, p0 + 9]
+    rows = st.active_rows(2)
+    assert rows[:8].tolist() == win.tolist() and sorted(rows[8:].tolist()) == [p0 + 1, p0 + 4]
+    assert len(set(rows.tolist())) == rows.size
