@@ -256,11 +256,13 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             for (int k = 0; k < kMaxActive / 32; ++k) {
                 const int i = k * 32 + lane;
                 posv[k] = -1;
+                if (k * 32 >= p.n_active) continue;   // uniform: nothing of the list left
                 if (i < p.n_active) posv[k] = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
             }
             int n_mine = 0, hi_tile = -1, lo_tile = T;   // last / first local tile that holds a refreshed position
 #pragma unroll
             for (int k = 0; k < kMaxActive / 32; ++k) {
+                if (k * 32 >= p.n_active) break;
                 const bool hit = posv[k] >= key_lo && posv[k] < key_hi;
                 const unsigned mk = __ballot_sync(0xffffffffu, hit);
                 if (hit) {
@@ -278,6 +280,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             int j_ref = T;
 #pragma unroll
             for (int k = 0; k < kMaxActive / 32; ++k) {
+                if (k * 32 >= p.n_active) break;
                 if (posv[k] >= key_lo && posv[k] < key_hi) {
                     const int tile = (posv[k] - key_lo) / BK;
                     int j;
