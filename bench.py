@@ -45,14 +45,14 @@ DEFAULT_WORKLOAD = "c2_llada_l768"
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
     "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-                    "sha256": "67630f6ddfc00b24fc9a8d18dbd9a73fbdcddf9dc0826592d3327fa6a0c71360",
-                    "bytes_per_launch": {"c2_llada_l768": 12965632, "c5_llada_l4096": 68294400}},
+                    "sha256": "088bb5de06a0d4a850fbc1673006a7b0cda103ce5b1fda2cdf38c16af0f2bfe9",
+                    "bytes_per_launch": {"c2_llada_l768": 12968960, "c5_llada_l4096": 68200704}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
                      "sha256": "5904bb11f13265705d4e4f6ec7dd6af483762e10fe0d7d597d0c44524eb63616",
                      "bytes_per_launch": {"c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
     "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
-                     "sha256": "08db22804ea2a9ba21796a5779146a48da833acacebe4fcd94b12ec2ec51e273",
-                     "bytes_per_launch": {"c5_llada_l4096_b8": 65467904}},
+                     "sha256": "7d578bb920ed3bc65f911bb747e22b6bb333a6dfcdf62f16dc30489f58ce07e4",
+                     "bytes_per_launch": {"c5_llada_l4096_b8": 65172992}},
 }
 
 
