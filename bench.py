@@ -49,10 +49,10 @@ NCU_TRAFFIC = {
                     "bytes_per_launch": {"c2_llada_l768": 12968960, "c5_llada_l4096": 68200704}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
                      "sha256": "5904bb11f13265705d4e4f6ec7dd6af483762e10fe0d7d597d0c44524eb63616",
-                     "bytes_per_launch": {"c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
+                     "bytes_per_launch": {"c2_llada_l768": 18928128, "c4_llada_l2048": 60842752, "c5_llada_l4096": 161536000}},
     "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
                      "sha256": "7d578bb920ed3bc65f911bb747e22b6bb333a6dfcdf62f16dc30489f58ce07e4",
-                     "bytes_per_launch": {"c5_llada_l4096_b8": 65172992}},
+                     "bytes_per_launch": {"c2_llada_l768": 8160768, "c5_llada_l4096_b8": 65172992}},
 }
 
 
