@@ -113,11 +113,13 @@ struct DenseParams {
     uint4* v_dst;
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
+    int q_tma;   // 1: one query head per kv head, the producer fetches the Q tiles with one TMA box each
     float scale_log2;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const DenseParams p) {
+attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                    const __grid_constant__ CUtensorMap map_q, const DenseParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (s2u(smem_raw) + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - s2u(smem_raw));
@@ -142,7 +144,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         prefetch_map(&map_k);
         prefetch_map(&map_v);
         for (int i = 0; i < B_COUNT; ++i)
-            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 256u : (i == B_QFULL ? (uint32_t)kSoftThreads : 1u));
+            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 256u : (i == B_QFULL && !p.q_tma ? (uint32_t)kSoftThreads : 1u));
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -161,6 +163,12 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (warp == 0) {
         // ================================ TMA producer ======================================
         if (lane == 0) {
+            if (p.q_tma) {   // Q first: [half][row][64 columns] per row tile; rows past n_active read as zero
+                prefetch_map(&map_q);
+                mbar_expect_tx(bar(B_QFULL), (uint32_t)n_tiles_q * TILE);
+                for (int t = 0; t < n_tiles_q; ++t)
+                    tma_load_5d(base + OFF_Q + t * TILE, &map_q, 0, r_pair + t * BM, hk, 0, b, bar(B_QFULL));
+            }
             for (int n = 0; n < 2 * T; ++n) {   // ring index: K_j = 2j, V_j = 2j + 1
                 const int slot = n % kSlots, u = n / kSlots;
                 if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
@@ -209,22 +217,24 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     } else if (warp < 2 + kSoftThreads / 32) {
         // ====================== Q staging, then softmax (warps 2..17) ========================
         const int stid = tid - 64;
-        // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
-        for (int c = stid; c < 2 * BM * (HD / 8); c += kSoftThreads) {
-            const int row = c >> 4, ch = c & 15;   // row in [0, 256)
-            const int r = r_pair + row;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < p.rows_total) {
-                const int i = r / p.group, j = r % p.group;
-                v = __ldg(reinterpret_cast<const uint4*>(
-                    p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + j) * HD + ch * 8));
+        if (!p.q_tma) {
+            // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
+            for (int c = stid; c < 2 * BM * (HD / 8); c += kSoftThreads) {
+                const int row = c >> 4, ch = c & 15;   // row in [0, 256)
+                const int r = r_pair + row;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (r < p.rows_total) {
+                    const int i = r / p.group, j = r % p.group;
+                    v = __ldg(reinterpret_cast<const uint4*>(
+                        p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + j) * HD + ch * 8));
+                }
+                const int t = row >> 7, rt = row & 127;
+                const uint32_t off = OFF_Q + t * TILE + (ch >> 3) * SUB + (rt >> 3) * 1024 + (rt & 7) * 128 + (((ch & 7) ^ (rt & 7)) << 4);
+                *reinterpret_cast<uint4*>(gbase + off) = v;
             }
-            const int t = row >> 7, rt = row & 127;
-            const uint32_t off = OFF_Q + t * TILE + (ch >> 3) * SUB + (rt >> 3) * 1024 + (rt & 7) * 128 + (((ch & 7) ^ (rt & 7)) << 4);
-            *reinterpret_cast<uint4*>(gbase + off) = v;
+            fence_async_smem();   // generic-proxy writes of Q -> visible to the tensor core (async proxy)
+            mbar_arrive(bar(B_QFULL));
         }
-        fence_async_smem();   // generic-proxy writes of Q -> visible to the tensor core (async proxy)
-        mbar_arrive(bar(B_QFULL));
 
         // A row of a tile is shared by two threads, one per 64-column half, in warps that own the same TMEM
         // lanes: softmax warp ws = warp - 2 -> row tile ws / 8, column half (ws / 4) % 2, lanes 32 * (warp % 4).
@@ -385,6 +395,8 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 }
 
 // ---- host side ---------------------------------------------------------------------------
+// Q of an MHA step seen as 5-D {64 columns, active row, head, half, sequence}: one box {64, 128, 1, 2, 1} lands as the
+// two 128-byte-swizzled halves of a [128 rows x 128] tile; rows past n_active read as zero.
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -454,6 +466,21 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     p.group = a.d.n_q_heads / a.d.n_kv_heads;
     p.rows_total = a.n_active * p.group;
     p.scale_log2 = a.scale * kLog2e;
+    p.q_tma = (p.group == 1) ? 1 : 0;
+    CUtensorMap map_q = map_k;   // unused unless q_tma
+    if (p.q_tma) {
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return cudaErrorInvalidValue;
+        const cuuint64_t dims[5] = {64, (cuuint64_t)a.n_active, (cuuint64_t)a.d.n_q_heads, 2, (cuuint64_t)a.d.batch};
+        const cuuint64_t strides[4] = {(cuuint64_t)a.d.n_q_heads * HD * 2, (cuuint64_t)HD * 2, 128,
+                                       (cuuint64_t)a.n_active * a.d.n_q_heads * HD * 2};
+        const cuuint32_t box[5] = {64, (cuuint32_t)BM, 1, 2, 1};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        if (fn(&map_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(a.q), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     static bool attr_done[64] = {};   // the attribute is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
@@ -472,7 +499,7 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, attend_dense_kernel, map_k, map_v, p);
+    return cudaLaunchKernelEx(&cfg, attend_dense_kernel, map_k, map_v, map_q, p);
 }
 
 }  // namespace ec
