@@ -262,7 +262,7 @@ def _graph_time(torch, body, replays: int, warmup: int, stream) -> float:
 
 def _workload(args) -> syn.Workload:
     """The named workload, with the recent-token budget replaced when --k-recent is given (the paper's default is
-    k = 64 and its grid 16..256; BASELINE's configurations use 1..8)."""
+    k = 64 and its grid 16..256; the named workloads use 2)."""
     import dataclasses
 
     w = syn.WORKLOADS[args.workload]
