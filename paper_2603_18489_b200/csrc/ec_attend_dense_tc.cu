@@ -6,7 +6,9 @@
 // TWO 128-row tiles of the packed (active row x query heads of one kv head) axis and walks over all
 // 128-key tiles of that kv head; while the softmax of one row tile runs, the tensor core works for the other.
 //   warp 0      TMA producer: K and V tiles ([128 keys x 128] bf16, one 4-D box each: [2 halves][128 keys]
-//               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...);
+//               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...); with one
+//               query head per kv head also the two Q tiles, one box each (otherwise the softmax warps stage
+//               them: the rows of a GQA tile interleave heads and positions, which no single box describes);
 //   warp 1      tcgen05.mma issuer (one thread): S_t = Q_t K^T (both operands K-major in shared memory) into
 //               the TMEM columns of row tile t, and O_t += P_t V with P_t read from TENSOR MEMORY (it
 //               overwrites the first 64 columns of S_t as packed bf16) and V MN-major from shared memory.
@@ -215,7 +217,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
         }
     } else if (warp < 2 + kSoftThreads / 32) {
-        // ====================== Q staging, then softmax (warps 2..17) ========================
+        // ============== Q staging (GQA shapes only), then softmax (warps 2..17) ===============
         const int stid = tid - 64;
         if (!p.q_tma) {
             // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)

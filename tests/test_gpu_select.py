@@ -55,6 +55,18 @@ def test_multi_step_traces_match_the_oracle(B, L, block, k):
     _trace(B, L, block, k, n_steps=40, seed=17 * L + k, n_cap=block + 256)
 
 
+def test_longest_supported_context_and_one_beyond():
+    """16384 positions (64 history entries per thread) is the limit; one more is refused by the host."""
+    import paper_2603_18489_b200 as ec
+
+    _trace(1, 16384, 32, 64, n_steps=12, seed=3, n_cap=32 + 128)
+    dev = torch.device("cuda")
+    z = torch.zeros(1, dtype=torch.int32, device=dev)
+    with pytest.raises(ec.EcError):
+        ec.ec_select_recent(ec.new_history(1, 16385), ec.new_step_state(1), torch.zeros(32, dtype=torch.uint8, device=dev),
+                            z, 32, z, 2, torch.empty(1, 64, dtype=torch.int32, device=dev))
+
+
 def test_row_list_is_cut_at_the_capacity_and_the_count_still_reports_the_need():
     _trace(2, 1024, 32, 64, n_steps=30, seed=5, n_cap=40, per_step_max=12)
 
