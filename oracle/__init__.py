@@ -260,3 +260,26 @@ def gate_metrics(entropy: np.ndarray, conf: np.ndarray, decoded_flags: np.ndarra
             out["entropy_sum"][b] = e[sl][d].sum()
             out["max_conf"][b] = c[sl][d].max()
     return out
+
+
+# --------------------------------------------------------------------------- #
+# Sliding-window decoding (Section 2.1; the paper's evaluation mode, window size 32).
+# --------------------------------------------------------------------------- #
+def sliding_window_rows(masked: np.ndarray, window: int) -> np.ndarray:
+    """The window of a step: the first `window` still-masked positions, ascending (fewer when fewer remain), so
+    that the number of masked tokens being denoised stays constant while the window advances over the sequence."""
+    return np.flatnonzero(np.asarray(masked) != 0)[:window].astype(np.int64)
+
+
+def sliding_step_bookkeeping(H: np.ndarray, masked: np.ndarray, t: int, dt: int, window_rows: np.ndarray,
+                             decoded_flags: np.ndarray, decision: int, k: int, window: int):
+    """Appendix A's statements after the decode of step t, with the mask tokens M given by a sliding window:
+    the flagged rows of the current window are decoded (H <- t, mask cleared), R follows Eq. 3, then skip_flag / dt / t,
+    then the next window.  H and masked are updated in place.  Returns (rows of the next partial step = next window
+    followed by R ascending, skip_flag, dt_next, t_next); the window and R are disjoint because R holds decoded
+    positions only."""
+    pos = np.asarray(window_rows, dtype=np.int64)[np.asarray(decoded_flags)[:len(window_rows)] != 0]
+    masked[pos] = 0
+    R, skip_flag, dt_next, t_next = step_bookkeeping(H, t, dt, pos, decision, k)
+    nxt = sliding_window_rows(masked, window)
+    return np.concatenate([nxt, R]), skip_flag, dt_next, t_next

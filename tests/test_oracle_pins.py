@@ -575,3 +575,41 @@ def test_gate_metrics_agree_with_the_gate_and_with_each_other():
         assert 1.0 / V <= m["max_conf"][b] <= 1.0
         # the most confident decoded row has at most -ln(conf) ... entropy bound from below: H >= -ln(max p)
         assert m["max_entropy"][b] >= -math.log(m["max_conf"][b]) - 1e-12 or n > 1
+
+
+# --------------------------------------------------------------------------- #
+# Sliding-window decoding (Section 2.1)
+# --------------------------------------------------------------------------- #
+def test_sliding_window_advances_and_keeps_its_size():
+    masked = np.array([0, 0, 1, 1, 1, 1, 1, 1, 1, 1], np.uint8)           # two prompt positions, eight to generate
+    H = np.full(10, -np.inf)
+    win = oracle.sliding_window_rows(masked, 4)
+    assert win.tolist() == [2, 3, 4, 5]
+    # step 1: rows 1 and 3 of the window (positions 3 and 5) are decoded; gate says skip
+    rows, skip, dt, t = oracle.sliding_step_bookkeeping(H, masked, 1, 0, win, np.array([0, 1, 0, 1], np.uint8), oracle.SKIP, 2, 4)
+    assert masked.tolist() == [0, 0, 1, 0, 1, 0, 1, 1, 1, 1] and H[3] == 1 and H[5] == 1
+    assert rows.tolist() == [2, 4, 6, 7, 3, 5] and skip and dt == 1 and t == 2      # window no longer contiguous, then R
+    # step 2: row 0 (position 2) decoded; K = {2 (H = 2), one of H = 1}, min 1, tau_R = max(1, 2 - 1) = 1
+    rows, skip, dt, t = oracle.sliding_step_bookkeeping(H, masked, t, dt, rows[:4], np.array([1, 0, 0, 0], np.uint8), oracle.SKIP, 2, 4)
+    assert rows.tolist() == [4, 6, 7, 8, 2, 3, 5] and dt == 2
+    # near the end fewer masked positions remain than the window holds
+    masked[:] = 0
+    masked[9] = 1
+    assert oracle.sliding_window_rows(masked, 4).tolist() == [9]
+
+
+def test_sliding_window_and_recent_set_never_overlap():
+    rng = np.random.Generator(np.random.PCG64(91))
+    L, window, k = 200, 16, 5
+    masked = np.ones(L, np.uint8); masked[:40] = 0
+    H = np.full(L, -np.inf)
+    t, dt = 1, 0
+    rows = oracle.sliding_window_rows(masked, window)
+    for step in range(12):
+        flags = (rng.random(window) < 0.25).astype(np.uint8)
+        win = rows[:window]
+        rows, skip, dt, t = oracle.sliding_step_bookkeeping(H, masked, t, dt, win, flags, int(rng.integers(0, 2)), k, window)
+        nxt, R = rows[:window], rows[window:]
+        assert nxt.size == window and np.all(np.diff(nxt) > 0) and np.all(masked[nxt] == 1)
+        assert np.all(np.isfinite(H[R])) and not set(nxt.tolist()) & set(R.tolist())
+        assert int(masked.sum()) == 160 - int(np.isfinite(H).sum())
