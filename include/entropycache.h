@@ -234,6 +234,24 @@ ec_status ec_select_recent(int32_t *history, int32_t ctx_len, int32_t batch, ec_
                            const int32_t *decision, int32_t k, int32_t *active_idx, int32_t n_cap,
                            void *stream);
 
+/* ec_select_recent for sliding-window decoding (Section 2.1 of the paper; its evaluation mode, window size 32): the
+ * window of a step is the first `window` still-masked positions of the sequence, so the number of mask tokens being
+ * denoised stays constant while the window advances; it stops being contiguous as soon as a position inside it is
+ * decoded.  Per sequence b, in one launch:
+ *   1. for every r < window with decoded_flags[b*window + r] != 0: pos = active_idx[b, r] (the window the previous
+ *      call wrote; before the first call the caller writes the first window there): history[b, pos] = t_b and
+ *      masked[b, pos] = 0                                                                      (Eq. 2)
+ *   2. K, tau_R, R exactly as ec_select_recent                                                 (Eq. 3)
+ *   3. skip_flag_b, dt_b, t_b exactly as ec_select_recent                                      (Appendix A)
+ *   4. active_idx[b, :] = the first `window` positions with masked[b, pos] != 0, ascending (fewer when fewer
+ *      remain), then the positions of R ascending (a decoded position is never masked, so the two are disjoint),
+ *      then -1 up to n_cap; state[b].n_active = their count (beyond n_cap the list is cut, as in ec_select_recent).
+ * masked: uint8 [batch, ctx_len], in/out; the other arguments as for ec_select_recent. */
+ec_status ec_select_recent_sliding(int32_t *history, int32_t ctx_len, int32_t batch, ec_step_state *state,
+                                   uint8_t *masked, const uint8_t *decoded_flags, int32_t window,
+                                   const int32_t *decision, int32_t k, int32_t *active_idx, int32_t n_cap,
+                                   void *stream);
+
 /* Zero-fills a workspace (asynchronous on `stream`). */
 ec_status ec_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 

@@ -70,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.ec_entropy_gate_decode.restype = i32
     lib.ec_select_recent.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, i32, vp, i32, vp]
     lib.ec_select_recent.restype = i32
+    lib.ec_select_recent_sliding.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, i32, vp, i32, vp]
+    lib.ec_select_recent_sliding.restype = i32
     lib.ec_workspace_init.argtypes = [vp, sz, vp]
     lib.ec_workspace_init.restype = i32
     lib.ec_status_string.argtypes = [i32]
@@ -323,3 +325,23 @@ def ec_entropy_gate_metrics(logits, vocab: int, rows_per_seq: int, decoded_flags
                                        workspace.numel() * workspace.element_size(), _stream(stream)),
            "ec_entropy_gate_metrics")
     return out
+
+
+def ec_select_recent_sliding(history, state, masked, decoded_flags, window: int, decision, k: int, active_idx,
+                             stream=None) -> None:
+    """ec_select_recent for sliding-window decoding (argument marshalling only).  masked uint8 [B, L] (in/out);
+    active_idx int32 [B, n_cap] holds the current window in its first `window` entries on entry and the next row
+    list on return."""
+    batch, ctx_len = history.shape
+    if history.dtype != torch.int32 or state.dtype != torch.int32 or active_idx.dtype != torch.int32:
+        raise TypeError("history, state and active_idx must be int32")
+    if masked.dtype != torch.uint8 or decoded_flags.dtype != torch.uint8 or decision.dtype != torch.int32:
+        raise TypeError("masked and decoded_flags must be uint8, decision int32")
+    if tuple(masked.shape) != (batch, ctx_len) or tuple(state.shape) != (batch, 4) or active_idx.shape[0] != batch:
+        raise ValueError("masked must be [B, L], state [B, 4], active_idx [B, n_cap]")
+    if decoded_flags.numel() != batch * window or decision.numel() != batch:
+        raise ValueError("decoded_flags must be [B * window], decision [B]")
+    _check(lib.ec_select_recent_sliding(_dev(history, "history"), int(ctx_len), int(batch), _dev(state, "state"),
+                                        _dev(masked, "masked"), _dev(decoded_flags, "decoded_flags"), int(window),
+                                        _dev(decision, "decision"), int(k), _dev(active_idx, "active_idx"),
+                                        int(active_idx.shape[1]), _stream(stream)), "ec_select_recent_sliding")

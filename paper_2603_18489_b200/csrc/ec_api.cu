@@ -103,7 +103,19 @@ ec_status ec_select_recent(int32_t* history, int32_t ctx_len, int32_t batch, ec_
         return EC_ERR_SHAPE;
     if (ctx_len > select_recent_max_ctx() || batch > 65535) return EC_ERR_UNSUPPORTED;
     const cudaError_t e = launch_select_recent(history, ctx_len, batch, state, decoded_flags, window_start, block,
-                                               decision, k, active_idx, n_cap, static_cast<cudaStream_t>(stream));
+                                               decision, k, active_idx, n_cap, nullptr, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+ec_status ec_select_recent_sliding(int32_t* history, int32_t ctx_len, int32_t batch, ec_step_state* state,
+                                   uint8_t* masked, const uint8_t* decoded_flags, int32_t window,
+                                   const int32_t* decision, int32_t k, int32_t* active_idx, int32_t n_cap, void* stream) {
+    if (!history || !state || !masked || !decoded_flags || !decision || !active_idx) return EC_ERR_NULL;
+    if (ctx_len < 1 || batch < 1 || window < 1 || window > ctx_len || k < 0 || k > ctx_len || n_cap < window)
+        return EC_ERR_SHAPE;
+    if (ctx_len > select_recent_max_ctx() || batch > 65535) return EC_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_select_recent(history, ctx_len, batch, state, decoded_flags, nullptr, window, decision, k,
+                                               active_idx, n_cap, masked, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
 }
 

@@ -61,7 +61,7 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream);
 int select_recent_max_ctx();
 cudaError_t launch_select_recent(int32_t* history, int ctx_len, int batch, ec_step_state* state, const uint8_t* decoded,
                                  const int32_t* window_start, int block, const int32_t* decision, int k,
-                                 int32_t* active_idx, int n_cap, cudaStream_t stream);
+                                 int32_t* active_idx, int n_cap, uint8_t* masked, cudaStream_t stream);
 
 cudaError_t launch_refresh(const ec_attn_desc& d, void* k_cache, void* v_cache, const void* k_new,
                            const void* v_new, const int32_t* active_idx, int n_active,

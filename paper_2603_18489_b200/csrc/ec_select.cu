@@ -23,6 +23,7 @@ struct SelectParams {
     const int32_t* window_start;
     const int32_t* decision;
     int32_t* active_idx;
+    uint8_t* masked;   // sliding-window mode: [batch, ctx_len] positions still masked (in/out); nullptr: block mode
     int ctx_len, block, k, n_cap;
 };
 
@@ -45,14 +46,39 @@ __global__ void __launch_bounds__(kSelThreads) select_recent_kernel(const Select
     const int b = blockIdx.x, tid = threadIdx.x;
     int32_t* H = p.history + (long long)b * p.ctx_len;
     ec_step_state st = p.state[b];
-    const int w0 = p.window_start[b];
-    if (w0 < 0 || w0 > p.ctx_len - p.block) {   // uniform over the CTA
+    const bool sliding = p.masked != nullptr;
+    uint8_t* M = sliding ? p.masked + (long long)b * p.ctx_len : nullptr;
+    int32_t* idx = p.active_idx + (long long)b * p.n_cap;
+    const int w0 = sliding ? 0 : p.window_start[b];
+    if (!sliding && (w0 < 0 || w0 > p.ctx_len - p.block)) {   // uniform over the CTA
         if (tid == 0) p.state[b].n_active = -1;
         return;
     }
+    // sliding mode: the current window holds min(block, masked positions left) rows; the list entries behind it are
+    // recent rows, not window rows, whatever their flags say
+    int n_cur = p.block;
+    if (sliding) {
+        const int per0 = (p.ctx_len + kSelThreads - 1) / kSelThreads;
+        int c = 0;
+        for (int j = 0; j < per0; ++j) {
+            const int pos = tid * per0 + j;
+            c += (pos < p.ctx_len && M[pos] != 0) ? 1 : 0;
+        }
+        c = block_sum(c, scratch);
+        n_cur = c < p.block ? c : p.block;
+        __syncthreads();
+    }
     // ---- Eq. 2: the positions decoded in this step get the step's index -----------------------------
-    for (int r = tid; r < p.block; r += kSelThreads)
-        if (p.decoded[(long long)b * p.block + r]) H[w0 + r] = st.t;
+    // block mode: window row r is position w0 + r; sliding mode: it is entry r of the row list of the previous call
+    for (int r = tid; r < n_cur; r += kSelThreads) {
+        if (p.decoded[(long long)b * p.block + r]) {
+            const int pos = sliding ? idx[r] : w0 + r;
+            if (pos >= 0 && pos < p.ctx_len) {
+                H[pos] = st.t;
+                if (sliding) M[pos] = 0;
+            }
+        }
+    }
     __syncthreads();
 
     const int per = (p.ctx_len + kSelThreads - 1) / kSelThreads;
@@ -99,58 +125,90 @@ __global__ void __launch_bounds__(kSelThreads) select_recent_kernel(const Select
             tau = tau > lo ? tau : lo;
         }
     }
-    // ---- R outside the block, ascending: per-thread counts, exclusive scan, compaction --------------
+    // exclusive scan of per-thread counts over the CTA (threads own ascending position ranges): base of this thread, total
+    const int lane = tid & 31, warp = tid >> 5;
+    auto block_scan = [&](int mine, int& base, int& total) {
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        __syncthreads();
+        if (lane == 31) scratch[warp] = incl;
+        __syncthreads();
+        if (tid == 0) {
+            int run = 0;
+            for (int w = 0; w < kSelThreads / 32; ++w) {
+                warp_base[w] = run;
+                run += scratch[w];
+            }
+            scratch[0] = run;
+        }
+        __syncthreads();
+        total = scratch[0];
+        base = warp_base[warp] + incl - mine;
+    };
+    // ---- the window's rows ---------------------------------------------------------------------------
+    int n_win = p.block;
+    if (!sliding) {
+        for (int r = tid; r < p.block; r += kSelThreads) idx[r] = w0 + r;   // block <= n_cap (checked on the host)
+    } else {
+        // sliding window: the first `block` positions that are still masked (fewer when fewer remain)
+        unsigned long long mbits = 0ull;
+        int mine_m = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int pos = i0 + j;
+            if (j < per && pos < p.ctx_len && M[pos] != 0) {
+                mbits |= 1ull << j;
+                ++mine_m;
+            }
+        }
+        int base_m, total_m;
+        block_scan(mine_m, base_m, total_m);
+        n_win = total_m < p.block ? total_m : p.block;
+        int at_m = base_m;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if ((mbits >> j) & 1ull) {
+                if (at_m < p.block) idx[at_m] = i0 + j;
+                ++at_m;
+            }
+        }
+    }
+    // ---- R (outside the block in block mode; a decoded position is never in a sliding window), ascending ----
     int mine = 0;
     if (!empty) {
 #pragma unroll
         for (int j = 0; j < PER; ++j) {
             const int pos = i0 + j;
             const bool in_r = h[j] != EC_H_NEVER && (long long)h[j] >= tau;
-            mine += (in_r && (pos < w0 || pos >= w0 + p.block)) ? 1 : 0;
+            mine += (in_r && (sliding || pos < w0 || pos >= w0 + p.block)) ? 1 : 0;
         }
     }
-    const int lane = tid & 31, warp = tid >> 5;
-    int incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
-    }
-    __syncthreads();
-    if (lane == 31) scratch[warp] = incl;
-    __syncthreads();
-    if (tid == 0) {
-        int run = 0;
-        for (int w = 0; w < kSelThreads / 32; ++w) {
-            warp_base[w] = run;
-            run += scratch[w];
-        }
-        scratch[0] = run;   // |R outside the block|
-    }
-    __syncthreads();
-    const int n_out = scratch[0];
-    int32_t* idx = p.active_idx + (long long)b * p.n_cap;
-    for (int r = tid; r < p.block; r += kSelThreads) idx[r] = w0 + r;   // block <= n_cap (checked on the host)
-    int at = p.block + warp_base[warp] + incl - mine;
+    int base_r, n_out;
+    block_scan(mine, base_r, n_out);
+    int at = n_win + base_r;
     if (!empty) {
 #pragma unroll
         for (int j = 0; j < PER; ++j) {
             const int pos = i0 + j;
             const bool in_r = h[j] != EC_H_NEVER && (long long)h[j] >= tau;
-            if (in_r && (pos < w0 || pos >= w0 + p.block)) {
+            if (in_r && (sliding || pos < w0 || pos >= w0 + p.block)) {
                 if (at < p.n_cap) idx[at] = pos;
                 ++at;
             }
         }
     }
-    for (int r = p.block + n_out + tid; r < p.n_cap; r += kSelThreads) idx[r] = -1;
+    for (int r = n_win + n_out + tid; r < p.n_cap; r += kSelThreads) idx[r] = -1;
     // ---- Appendix A: skip_flag, dt, t ------------------------------------------------------------------
     if (tid == 0) {
         const int skip = p.decision[b] == EC_SKIP ? 1 : 0;
         st.skip_flag = skip;
         st.dt_recompute = skip ? st.dt_recompute + 1 : 0;
         st.t = st.t + 1;
-        st.n_active = p.block + n_out;
+        st.n_active = n_win + n_out;
         p.state[b] = st;
     }
 }
@@ -161,8 +219,8 @@ int select_recent_max_ctx() { return kSelMaxPer * kSelThreads; }
 
 cudaError_t launch_select_recent(int32_t* history, int ctx_len, int batch, ec_step_state* state, const uint8_t* decoded,
                                  const int32_t* window_start, int block, const int32_t* decision, int k,
-                                 int32_t* active_idx, int n_cap, cudaStream_t stream) {
-    SelectParams p{history, state, decoded, window_start, decision, active_idx, ctx_len, block, k, n_cap};
+                                 int32_t* active_idx, int n_cap, uint8_t* masked, cudaStream_t stream) {
+    SelectParams p{history, state, decoded, window_start, decision, active_idx, masked, ctx_len, block, k, n_cap};
     if (ctx_len <= 4 * kSelThreads) select_recent_kernel<4><<<batch, kSelThreads, 0, stream>>>(p);
     else if (ctx_len <= 16 * kSelThreads) select_recent_kernel<16><<<batch, kSelThreads, 0, stream>>>(p);
     else select_recent_kernel<kSelMaxPer><<<batch, kSelThreads, 0, stream>>>(p);

@@ -103,3 +103,50 @@ def test_argument_errors_are_reported_by_the_host():
         ec.ec_select_recent(hist, state, flags, z, 32, z, 129, torch.empty(1, 64, dtype=torch.int32, device=dev))   # k > L
     with pytest.raises(ec.EcError):
         ec.ec_select_recent(hist, state, flags, z, 32, z, 2, torch.empty(1, 16, dtype=torch.int32, device=dev))    # n_cap < block
+
+
+def _sliding_trace(B, L, prompt, window, k, n_steps, seed, n_cap):
+    import paper_2603_18489_b200 as ec
+
+    rng = np.random.Generator(np.random.PCG64(seed))
+    dev = torch.device("cuda")
+    hist, state = ec.new_history(B, L), ec.new_step_state(B, 1)
+    masked_np = np.ones((B, L), np.uint8)
+    masked_np[:, :prompt] = 0
+    masked = torch.from_numpy(masked_np.copy()).to(dev)
+    idx = torch.full((B, n_cap), -1, dtype=torch.int32, device=dev)
+    H = [np.full(L, -np.inf) for _ in range(B)]
+    M = [masked_np[b].copy() for b in range(B)]
+    cur = [oracle.sliding_window_rows(M[b], window) for b in range(B)]      # the current window of each sequence
+    for b in range(B):                                                       # the caller seeds the first window
+        idx[b, :cur[b].size] = torch.from_numpy(cur[b].astype(np.int32)).to(dev)
+    t, dt = [1] * B, [0] * B
+    for s in range(n_steps):
+        flags = (rng.random((B, window)) < 0.2).astype(np.uint8)             # flags behind a shrunken window are ignored
+        dec = rng.integers(0, 2, size=B).astype(np.int32)
+        ec.ec_select_recent_sliding(hist, state, masked, torch.from_numpy(flags.reshape(-1)).to(dev), window,
+                                    torch.from_numpy(dec).to(dev), k, idx)
+        torch.cuda.synchronize()
+        g_hist, g_state, g_idx, g_m = hist.cpu().numpy(), state.cpu().numpy(), idx.cpu().numpy(), masked.cpu().numpy()
+        for b in range(B):
+            new_rows, skip, dt[b], t[b] = oracle.sliding_step_bookkeeping(H[b], M[b], t[b], dt[b], cur[b], flags[b],
+                                                                           int(dec[b]), k, window)
+            cur[b] = new_rows[:min(window, int(M[b].sum()))]
+            want_h = np.where(np.isfinite(H[b]), H[b], NEVER).astype(np.int64)
+            assert np.array_equal(g_hist[b].astype(np.int64), want_h), (s, b)
+            assert np.array_equal(g_m[b], M[b]), (s, b)
+            assert g_state[b].tolist() == [t[b], dt[b], int(skip), new_rows.size], (s, b)
+            n_keep = min(new_rows.size, n_cap)
+            assert g_idx[b, :n_keep].tolist() == new_rows[:n_keep].tolist(), (s, b)
+            assert np.all(g_idx[b, n_keep:] == -1)
+
+
+@pytest.mark.parametrize("B,L,prompt,window,k", [(1, 768, 512, 32, 2), (4, 4096, 3072, 32, 64), (2, 300, 100, 8, 3),
+                                                 (2, 1024, 0, 128, 16), (1, 6000, 5000, 32, 8)])
+def test_sliding_window_traces_match_the_oracle(B, L, prompt, window, k):
+    _sliding_trace(B, L, prompt, window, k, n_steps=30, seed=19 * L + k, n_cap=window + 512)
+
+
+def test_sliding_window_runs_out_of_masked_positions():
+    """40 positions to generate, window 16: after a few steps fewer than 16 remain and the window shrinks to what is left."""
+    _sliding_trace(1, 140, 100, 16, 4, n_steps=40, seed=77, n_cap=16 + 64)
