@@ -6,9 +6,10 @@
 // TWO 128-row tiles of the packed (active row x query heads of one kv head) axis and walks over all
 // 128-key tiles of that kv head; while the softmax of one row tile runs, the tensor core works for the other.
 //   warp 0      TMA producer: K and V tiles ([128 keys x 128] bf16, one 4-D box each: [2 halves][128 keys]
-//               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...); with one
-//               query head per kv head also the two Q tiles, one box each (otherwise the softmax warps stage
-//               them: the rows of a GQA tile interleave heads and positions, which no single box describes);
+//               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...), and the
+//               two Q tiles of the unit, one box each.  (Grouped-query shapes are launched with one unit per
+//               QUERY head, so a row tile is always 128 active rows of one head; the query heads of a kv head
+//               stream the same K/V, which L2 serves.  The thread-staged Q path below remains for packed tiles.)
 //   warp 1      tcgen05.mma issuer (one thread): S_t = Q_t K^T (both operands K-major in shared memory) into
 //               the TMEM columns of row tile t, and O_t += P_t V with P_t read from TENSOR MEMORY (it
 //               overwrites the first 64 columns of S_t as packed bf16) and V MN-major from shared memory.
@@ -116,6 +117,10 @@ struct DenseParams {
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
     int q_tma;   // 1: one query head per kv head, the producer fetches the Q tiles with one TMA box each
+    // Grouped-query shapes run with one unit per QUERY head (the kernel then sees n_kv_heads = n_q_heads = H_q and
+    // group = 1, so its row tiles are 128 active rows of one head and come by TMA); the K/V of unit head h are
+    // those of the real kv head h / kv_div, of which there are n_kv_real.  kv_div = 1 otherwise.
+    int kv_div, n_kv_real;
     float scale_log2;
 };
 
@@ -165,6 +170,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     if (warp == 0) {
         // ================================ TMA producer ======================================
         if (lane == 0) {
+            const int hk_kv = hk / p.kv_div;
             if (p.q_tma) {   // Q first: [half][row][64 columns] per row tile; rows past n_active read as zero
                 prefetch_map(&map_q);
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)n_tiles_q * TILE);
@@ -175,7 +181,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const int slot = n % kSlots, u = n / kSlots;
                 if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
                 mbar_expect_tx(bar(B_FULL + slot), TILE);
-                tma_load_5d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, hk, b, bar(B_FULL + slot));
+                tma_load_5d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, hk_kv, b, bar(B_FULL + slot));
             }
         }
     } else if (warp == 1) {
@@ -362,9 +368,11 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // The (row-tile pair, kv head) CTAs of a head split its positions evenly; a position's K and V rows
         // (256 bytes each) go from [b, pos, hk, :] to [b, hk, pos, :].  Two rows per warp instruction, eight
         // instructions in flight.  Nobody reads the cache in this launch.
-        const int n_pairs = gridDim.x;
-        const int per = (p.ctx_len + n_pairs - 1) / n_pairs;
-        const int pos0 = pair * per, pos1 = min(p.ctx_len, pos0 + per);
+        // (with one unit per query head, the kv_div units of a real kv head share its positions as well)
+        const int hk_kv = hk / p.kv_div;
+        const int n_share = gridDim.x * p.kv_div;
+        const int per = (p.ctx_len + n_share - 1) / n_share;
+        const int pos0 = ((hk % p.kv_div) * gridDim.x + pair) * per, pos1 = min(p.ctx_len, pos0 + per);
         const int sub = lane >> 4, piece = lane & 15;
         for (int pos = pos0; pos < pos1; pos += 16) {
             uint4 kv[8], vv[8];
@@ -372,7 +380,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             for (int u = 0; u < 8; ++u) {
                 const int pp = pos + 2 * u + sub;
                 if (pp < pos1) {
-                    const long long src = (((long long)b * p.ctx_len + pp) * p.n_kv_heads + hk) * 16 + piece;
+                    const long long src = (((long long)b * p.ctx_len + pp) * p.n_kv_real + hk_kv) * 16 + piece;
                     kv[u] = __ldg(p.k_src + src);
                     vv[u] = __ldg(p.v_src + src);
                 }
@@ -381,7 +389,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             for (int u = 0; u < 8; ++u) {
                 const int pp = pos + 2 * u + sub;
                 if (pp < pos1) {
-                    const long long dst = (((long long)b * p.n_kv_heads + hk) * p.ctx_len + pp) * 16 + piece;
+                    const long long dst = (((long long)b * p.n_kv_real + hk_kv) * p.ctx_len + pp) * 16 + piece;
                     p.k_dst[dst] = kv[u];
                     p.v_dst[dst] = vv[u];
                 }
@@ -439,15 +447,15 @@ bool make_kv_map(CUtensorMap* map, const void* ptr, int batch, int n_kv_heads, i
 // the two-tile kernel has no key split: it is used when the (row-tile pair, kv head) units fill the GPU
 bool attend_dense_supported(const ec_attn_desc& d, int n_active) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
-    const long long rows = (long long)n_active * (d.n_q_heads / d.n_kv_heads);
-    const long long pairs = (rows + 2 * BM - 1) / (2 * BM);
-    const long long bh = (long long)d.batch * d.n_kv_heads;
+    // one unit per (sequence, query head, row-tile pair): grouped-query shapes are run head by head
+    const long long pairs = ((long long)n_active + 2 * BM - 1) / (2 * BM);
+    const long long bh = (long long)d.batch * d.n_q_heads;
     if (bh > 65535 || pairs > 0x7fffffffLL) return false;
     return pairs * bh >= sm_count() / 2;
 }
 
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
-    const int bh = a.d.batch * a.d.n_kv_heads;
+    const int bh = a.d.batch * a.d.n_q_heads;
     CUtensorMap map_k, map_v;
     if (!make_kv_map(&map_k, a.k_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major) ||
         !make_kv_map(&map_v, a.v_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major))
@@ -464,11 +472,13 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     p.n_active = a.n_active;
     p.ctx_len = a.d.ctx_len;
     p.n_q_heads = a.d.n_q_heads;
-    p.n_kv_heads = a.d.n_kv_heads;
-    p.group = a.d.n_q_heads / a.d.n_kv_heads;
-    p.rows_total = a.n_active * p.group;
+    p.n_kv_heads = a.d.n_q_heads;   // the kernel's heads are the query heads, see kv_div
+    p.group = 1;
+    p.rows_total = a.n_active;
+    p.kv_div = a.d.n_q_heads / a.d.n_kv_heads;
+    p.n_kv_real = a.d.n_kv_heads;
     p.scale_log2 = a.scale * kLog2e;
-    p.q_tma = (p.group == 1) ? 1 : 0;
+    p.q_tma = 1;
     CUtensorMap map_q = map_k;   // unused unless q_tma
     if (p.q_tma) {
         EncodeTiledFn fn = encode_fn();
