@@ -48,8 +48,8 @@ NCU_TRAFFIC = {
                     "sha256": "088bb5de06a0d4a850fbc1673006a7b0cda103ce5b1fda2cdf38c16af0f2bfe9",
                     "bytes_per_launch": {"c2_llada_l768": 12968960, "c5_llada_l4096": 68200704}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
-                     "sha256": "b99c0896626a84951749b9d5c3d2cc6ec493926d7c8b7662365eb314fa523905",
-                     "bytes_per_launch": {"c2_llada_l768": 18925824, "c4_llada_l2048": 62815744, "c5_llada_l4096": 166534144}},
+                     "sha256": "54ec597014094429ac7064859b7b2ca2a2537ad8867d42cc57f9e8822b2caf58",
+                     "bytes_per_launch": {"c2_llada_l768": 18928896, "c4_llada_l2048": 60230144, "c5_llada_l4096": 161412864}},
     "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
                      "sha256": "7d578bb920ed3bc65f911bb747e22b6bb333a6dfcdf62f16dc30489f58ce07e4",
                      "bytes_per_launch": {"c2_llada_l768": 8160768, "c5_llada_l4096_b8": 65172992}},
