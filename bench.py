@@ -45,7 +45,7 @@ DEFAULT_WORKLOAD = "c2_llada_l768"
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
     "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-                    "sha256": "088bb5de06a0d4a850fbc1673006a7b0cda103ce5b1fda2cdf38c16af0f2bfe9",
+                    "sha256": "e9aff5110c7667b8ad12c758605c719f594430da1eacc5bb078ee95d7f223974",
                     "bytes_per_launch": {"c2_llada_l768": 12968960, "c5_llada_l4096": 68200704}},
     "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
                      "sha256": "54ec597014094429ac7064859b7b2ca2a2537ad8867d42cc57f9e8822b2caf58",

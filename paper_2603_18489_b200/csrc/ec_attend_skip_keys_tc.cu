@@ -774,7 +774,7 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
         return cudaErrorInvalidValue;
     KeysParams p{};
     CUtensorMap map_q = map_k;   // unused unless q_tma
-    p.q_tma = (a.d.n_q_heads == a.d.n_kv_heads) ? 1 : 0;
+    p.q_tma = (pl.group == 1) ? 1 : 0;   // one query head per CTA column: its rows are one TMA box
     if (p.q_tma && !make_q_map(&map_q, a.q, a.d.batch, a.n_active, a.d.n_q_heads, pl.n_slots)) return cudaErrorInvalidValue;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
