@@ -110,7 +110,10 @@ C4 = Workload(4, "c4_llada_l2048", BF16, 1, 32, 32, 128, 1024, 1024, 32, 2, 1264
 C5 = Workload(5, "c5_llada_l4096", BF16, 1, 32, 32, 128, 3072, 1024, 32, 2, 126464,
               n_layers=32, n_steps=64)
 C5B8 = replace(C5, name="c5_llada_l4096_b8", batch=8)
-WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, C5B8)}
+# the second model geometry of the paper's evaluation (Dream-7B: 28 query heads on 4 kv heads) at the long contexts
+C4D = Workload(6, "c4_dream_l2048", BF16, 1, 28, 4, 128, 1024, 1024, 32, 2, 152064, n_steps=32)
+C5D = Workload(7, "c5_dream_l4096", BF16, 1, 28, 4, 128, 3072, 1024, 32, 2, 152064, n_layers=28, n_steps=64)
+WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, C5B8, C4D, C5D)}
 BY_ID = {1: C1, 2: C2, 3: C3, 4: C4, 5: C5}
 
 # tensor ids for the seeding rule
@@ -152,6 +155,19 @@ def active_rows(w: Workload, block_no: int = 0, k_recent: int | None = None,
             rng.shuffle(row)
         out[b] = row
     return out
+
+
+def consecutive_runs(seq_ids) -> list[tuple[int, int]]:
+    """Maximal runs of consecutive sequence numbers in an ascending list, as (first, count) pairs:
+    [0, 1, 4] -> [(0, 2), (4, 1)].  A step in which the sequences of a batch took different decisions issues one
+    call per run of each kind (a run is a contiguous slice of every batch-major tensor)."""
+    runs = []
+    for b in seq_ids:
+        if runs and runs[-1][0] + runs[-1][1] == b:
+            runs[-1] = (runs[-1][0], runs[-1][1] + 1)
+        else:
+            runs.append((int(b), 1))
+    return runs
 
 
 # --------------------------------------------------------------------------- #

@@ -109,11 +109,22 @@ size_t ec_attend_workspace_bytes(const ec_attn_desc *desc, int32_t n_active);
  * k_new and v_new may both be NULL to attend without refreshing.  workspace: at
  * least ec_attend_workspace_bytes() bytes, 16-byte aligned, zero-filled before
  * first use.  dev_status (nullable, device int32): set to an ec_status by the
- * kernels if a bounded wait ran out; untouched otherwise. */
+ * kernels if a bounded wait ran out; untouched otherwise.  When *dev_status is non-zero after the call has
+ * completed, `out` and the refreshed cache rows of that call are unspecified: always pass dev_status where a
+ * wrong row must not go unnoticed (with NULL a timed-out step returns whatever it had computed). */
 ec_status ec_attend(const ec_attn_desc *desc, const void *q, const void *k_new, const void *v_new,
                     void *k_cache, void *v_cache, const int32_t *active_idx, int32_t n_active,
                     void *out, void *workspace, size_t workspace_bytes,
                     int32_t *dev_status, void *stream);
+
+/* (No counterpart in the paper: a host-only query for tests and reports.)
+ * Describes the launch ec_attend would make for this geometry: the kernel's name with its template instantiation,
+ * then "grid=(x,y) cluster=c ..." for the tensor-core kernels, e.g. "attend_skip_keys_kernel<48> grid=(4,32)
+ * cluster=4 stages=3 smem=...".  with_fresh_kv: k_new/v_new would be given; with_index_list: active_idx would be
+ * non-NULL.  Touches no device memory and launches nothing.  Returns "" on arguments ec_attend would reject.  The
+ * string lives in a thread-local buffer that the next call on the same thread overwrites. */
+const char *ec_attend_kernel_name(const ec_attn_desc *desc, int32_t n_active, int32_t with_fresh_kv,
+                                  int32_t with_index_list);
 
 /* Bytes of workspace ec_entropy_gate needs (0 on bad arguments). */
 size_t ec_entropy_gate_workspace_bytes(int32_t n_rows, int32_t vocab);

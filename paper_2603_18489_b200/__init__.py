@@ -56,6 +56,8 @@ def _load() -> ctypes.CDLL:
     lib.ec_attend_workspace_bytes.restype = sz
     lib.ec_attend.argtypes = [dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
     lib.ec_attend.restype = i32
+    lib.ec_attend_kernel_name.argtypes = [dp, i32, i32, i32]
+    lib.ec_attend_kernel_name.restype = ctypes.c_char_p
     lib.ec_entropy_gate_workspace_bytes.argtypes = [i32, i32]
     lib.ec_entropy_gate_workspace_bytes.restype = sz
     lib.ec_entropy_gate.argtypes = [vp, i32, i32, i32, i64, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -138,6 +140,12 @@ def new_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
 
 def ec_attend_workspace_bytes(desc: ec_attn_desc, n_active: int) -> int:
     return int(lib.ec_attend_workspace_bytes(ctypes.byref(desc), int(n_active)))
+
+
+def ec_attend_kernel_name(desc: ec_attn_desc, n_active: int, with_fresh_kv: bool = True,
+                          with_index_list: bool = True) -> str:
+    """Host-only: which kernel (and launch shape) ec_attend picks for this geometry."""
+    return lib.ec_attend_kernel_name(ctypes.byref(desc), int(n_active), int(with_fresh_kv), int(with_index_list)).decode()
 
 
 def ec_entropy_gate_workspace_bytes(n_rows: int, vocab: int) -> int:

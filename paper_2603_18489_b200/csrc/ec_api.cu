@@ -3,22 +3,29 @@
 #include "ec_common.cuh"
 
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
 namespace ec {
 
 int sm_count() {
-    static std::atomic<int> cached{0};
-    int v = cached.load(std::memory_order_relaxed);
-    if (v > 0) return v;
+    static std::atomic<int> cached[kMaxDevices] = {};   // per device ordinal: a process may drive unlike GPUs
     int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    if (cudaGetDevice(&dev) != cudaSuccess) {
         (void)cudaGetLastError();  // no device (host-only use of the size queries): not sticky
         return kDefaultSmCount;
     }
-    cached.store(n, std::memory_order_relaxed);
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    if (slot) {
+        const int v = cached[dev].load(std::memory_order_relaxed);
+        if (v > 0) return v;
+    }
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        return kDefaultSmCount;
+    }
+    if (slot) cached[dev].store(n, std::memory_order_relaxed);
     return n;
 }
 
@@ -56,6 +63,17 @@ size_t attend_ws(const ec_attn_desc& d, int n_active) {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// which kernel serves a call of ec_attend: the one place the dispatch order is written down
+enum AttendPath { PATH_SKIP_KEYS, PATH_SKIP_ROWS, PATH_DENSE_FROM_NEW, PATH_DENSE, PATH_TC_ONE_TILE, PATH_MMA, PATH_F32 };
+AttendPath choose_path(const ec_attn_desc& d, int n_active, bool fresh_kv, bool index_list) {
+    if (use_skip_keys(d, n_active)) return PATH_SKIP_KEYS;
+    if (use_skip(d, n_active)) return PATH_SKIP_ROWS;
+    if (d.dtype != EC_BF16) return PATH_F32;
+    if (use_tc(d) && forced_impl() != 2 && attend_dense_supported(d, n_active))
+        return fresh_kv && !index_list ? PATH_DENSE_FROM_NEW : PATH_DENSE;
+    return use_tc(d) ? PATH_TC_ONE_TILE : PATH_MMA;
+}
+
 ec_status check_desc(const ec_attn_desc* d) {
     if (!d) return EC_ERR_NULL;
     if (d->dtype != EC_F32 && d->dtype != EC_BF16) return EC_ERR_DTYPE;
@@ -75,6 +93,42 @@ ec_status check_active(const ec_attn_desc* d, const int32_t* active_idx, int32_t
 }
 
 }  // namespace
+}  // namespace ec
+
+namespace ec {
+
+// every host-side check of the gate entry points; EC_OK means a launch with these arguments is well-formed
+// (n_rows == 0 is EC_OK too: the callers return before launching)
+ec_status gate_validate(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride_elems,
+                        int32_t rows_per_seq, const uint8_t* decoded_flags, uint8_t* masked, float conf_threshold,
+                        uint8_t* decoded_out, int32_t* tokens, float tau, int32_t* argmax_out, float* conf_out,
+                        float* entropy_out, float* max_entropy_out, int32_t* decision_out, float* entropy_sum_out,
+                        float* max_conf_out, const void* workspace, size_t workspace_bytes) {
+    if (dtype != EC_F32 && dtype != EC_BF16) return EC_ERR_DTYPE;
+    if (n_rows < 0 || vocab < 1 || rows_per_seq < 1 || row_stride_elems < vocab) return EC_ERR_SHAPE;
+    if (n_rows % rows_per_seq != 0) return EC_ERR_SHAPE;
+    if (n_rows > 65535) return EC_ERR_UNSUPPORTED;          // grid.y limit
+    if (vocab > 96 * 8192) return EC_ERR_UNSUPPORTED;       // split table of the workspace
+    if (tau != tau) return EC_ERR_SHAPE;
+    const bool decode = masked != nullptr || decoded_out != nullptr || tokens != nullptr;
+    if (decode && (conf_threshold != conf_threshold)) return EC_ERR_SHAPE;
+    const bool one_cta_finish = decode || entropy_sum_out != nullptr || max_conf_out != nullptr;
+    if (one_cta_finish && rows_per_seq > kGateDecodeMaxRowsPerSeq) return EC_ERR_UNSUPPORTED;
+    if (n_rows == 0) return EC_OK;
+    if (!logits || !max_entropy_out || !decision_out) return EC_ERR_NULL;
+    if (decode ? (!masked || !decoded_out || !tokens) : !decoded_flags) return EC_ERR_NULL;
+    const size_t esize = dtype == EC_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(logits) & 15u) || ((size_t)row_stride_elems * esize) % 16 != 0) return EC_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(argmax_out) | reinterpret_cast<uintptr_t>(conf_out) |
+         reinterpret_cast<uintptr_t>(entropy_out) | reinterpret_cast<uintptr_t>(max_entropy_out) |
+         reinterpret_cast<uintptr_t>(decision_out) | reinterpret_cast<uintptr_t>(tokens) |
+         reinterpret_cast<uintptr_t>(entropy_sum_out) | reinterpret_cast<uintptr_t>(max_conf_out)) & 3u)
+        return EC_ERR_ALIGN;
+    const size_t need = gate_workspace_bytes(n_rows, vocab);
+    if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
+    return EC_OK;
+}
+
 }  // namespace ec
 
 using namespace ec;
@@ -142,13 +196,12 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
     if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
     if (!aligned16(workspace)) return EC_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool fused_keys = use_skip_keys(*desc, n_active);
-    const bool fused = fused_keys || use_skip(*desc, n_active);
-
-    const bool dense = !fused && use_tc(*desc) && forced_impl() != 2 && attend_dense_supported(*desc, n_active);
+    const AttendPath path = choose_path(*desc, n_active, k_new != nullptr, active_idx != nullptr);
+    const bool fused_keys = path == PATH_SKIP_KEYS;
+    const bool fused = fused_keys || path == PATH_SKIP_ROWS;
     // recompute step on the dense path: every cache row is overwritten by the fresh row of the same position, so
     // attention reads K/V straight from k_new / v_new and a spare warp of the same launch copies them into the cache
-    const bool from_new = dense && k_new && !active_idx;
+    const bool from_new = path == PATH_DENSE_FROM_NEW;
     if (k_new && !fused && !from_new) {
         if (launch_refresh(*desc, k_cache, v_cache, k_new, v_new, active_idx, n_active, s) != cudaSuccess)
             return EC_ERR_CUDA;
@@ -171,47 +224,57 @@ ec_status ec_attend(const ec_attn_desc* desc, const void* q, const void* k_new, 
         a.refresh_k_dst = k_cache;
         a.refresh_v_dst = v_cache;
     }
-    const cudaError_t e = fused_keys             ? launch_attend_skip_keys(a, k_new, v_new, active_idx, s)
-                          : fused                ? launch_attend_skip(a, k_new, v_new, active_idx, s)
-                          : desc->dtype != EC_BF16 ? launch_attend_f32(a, s)
-                          : dense                ? launch_attend_dense(a, s)
-                          : use_tc(*desc)        ? launch_attend_bf16_tc(a, s)
-                                                 : launch_attend_bf16(a, s);
+    cudaError_t e;
+    switch (path) {
+        case PATH_SKIP_KEYS: e = launch_attend_skip_keys(a, k_new, v_new, active_idx, s); break;
+        case PATH_SKIP_ROWS: e = launch_attend_skip(a, k_new, v_new, active_idx, s); break;
+        case PATH_F32: e = launch_attend_f32(a, s); break;
+        case PATH_DENSE_FROM_NEW:
+        case PATH_DENSE: e = launch_attend_dense(a, s); break;
+        case PATH_TC_ONE_TILE: e = launch_attend_bf16_tc(a, s); break;
+        default: e = launch_attend_bf16(a, s); break;
+    }
     return e == cudaSuccess ? EC_OK : EC_ERR_CUDA;
+}
+
+const char* ec_attend_kernel_name(const ec_attn_desc* desc, int32_t n_active, int32_t with_fresh_kv,
+                                  int32_t with_index_list) {
+    static thread_local char buf[192];
+    if (check_desc(desc) != EC_OK || n_active < 1 || n_active > desc->ctx_len ||
+        (!with_index_list && n_active != desc->ctx_len))
+        return "";
+    const bool fresh = with_fresh_kv != 0;
+    switch (choose_path(*desc, n_active, fresh, with_index_list != 0)) {
+        case PATH_SKIP_KEYS: attend_skip_keys_describe(*desc, n_active, buf, sizeof buf); return buf;
+        case PATH_SKIP_ROWS: attend_skip_describe(*desc, n_active, buf, sizeof buf); return buf;
+        case PATH_F32: return fresh ? "refresh_kernel + attend_f32_kernel" : "attend_f32_kernel";
+        case PATH_DENSE_FROM_NEW: attend_dense_describe(*desc, n_active, buf, sizeof buf); return buf;
+        case PATH_DENSE: {
+            char inner[160];
+            attend_dense_describe(*desc, n_active, inner, sizeof inner);
+            snprintf(buf, sizeof buf, "%s%s", fresh ? "refresh_kernel + " : "", inner);
+            return buf;
+        }
+        case PATH_TC_ONE_TILE: return fresh ? "refresh_kernel + attend_tc_kernel" : "attend_tc_kernel";
+        default: return fresh ? "refresh_kernel + attend_mma_kernel" : "attend_mma_kernel";
+    }
 }
 
 size_t ec_entropy_gate_workspace_bytes(int32_t n_rows, int32_t vocab) { return gate_workspace_bytes(n_rows, vocab); }
 
 namespace {
 
-// shared by ec_entropy_gate and ec_entropy_gate_decode: `masked` selects the decode mode
+// shared by ec_entropy_gate, ec_entropy_gate_metrics and ec_entropy_gate_decode: `masked` selects the decode mode
 ec_status gate_call(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride_elems,
                     int32_t rows_per_seq, const uint8_t* decoded_flags, uint8_t* masked, float conf_threshold,
                     uint8_t* decoded_out, int32_t* tokens, float tau, int32_t* argmax_out, float* conf_out,
                     float* entropy_out, float* max_entropy_out, int32_t* decision_out, float* entropy_sum_out,
                     float* max_conf_out, void* workspace, size_t workspace_bytes, void* stream) {
-    if (dtype != EC_F32 && dtype != EC_BF16) return EC_ERR_DTYPE;
-    if (n_rows < 0 || vocab < 1 || rows_per_seq < 1 || row_stride_elems < vocab) return EC_ERR_SHAPE;
-    if (n_rows % rows_per_seq != 0) return EC_ERR_SHAPE;
-    if (n_rows > 65535) return EC_ERR_UNSUPPORTED;          // grid.y limit
-    if (vocab > 96 * 8192) return EC_ERR_UNSUPPORTED;       // split table of the workspace
-    if (tau != tau) return EC_ERR_SHAPE;
-    const bool decode = masked != nullptr || decoded_out != nullptr || tokens != nullptr;
-    if (decode && (conf_threshold != conf_threshold)) return EC_ERR_SHAPE;
-    const bool one_cta_finish = decode || entropy_sum_out != nullptr || max_conf_out != nullptr;
-    if (one_cta_finish && rows_per_seq > kGateDecodeMaxRowsPerSeq) return EC_ERR_UNSUPPORTED;
-    if (n_rows == 0) return EC_OK;
-    if (!logits || !max_entropy_out || !decision_out) return EC_ERR_NULL;
-    if (decode ? (!masked || !decoded_out || !tokens) : !decoded_flags) return EC_ERR_NULL;
-    const size_t esize = dtype == EC_BF16 ? 2 : 4;
-    if (!aligned16(logits) || ((size_t)row_stride_elems * esize) % 16 != 0) return EC_ERR_ALIGN;
-    if ((reinterpret_cast<uintptr_t>(argmax_out) | reinterpret_cast<uintptr_t>(conf_out) |
-         reinterpret_cast<uintptr_t>(entropy_out) | reinterpret_cast<uintptr_t>(max_entropy_out) |
-         reinterpret_cast<uintptr_t>(decision_out) | reinterpret_cast<uintptr_t>(tokens) |
-         reinterpret_cast<uintptr_t>(entropy_sum_out) | reinterpret_cast<uintptr_t>(max_conf_out)) & 3u)
-        return EC_ERR_ALIGN;
-    const size_t need = gate_workspace_bytes(n_rows, vocab);
-    if (!workspace || workspace_bytes < need) return EC_ERR_WORKSPACE;
+    const ec_status st = gate_validate(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags, masked,
+                                       conf_threshold, decoded_out, tokens, tau, argmax_out, conf_out, entropy_out,
+                                       max_entropy_out, decision_out, entropy_sum_out, max_conf_out, workspace,
+                                       workspace_bytes);
+    if (st != EC_OK || n_rows == 0) return st;
     GateArgs a;
     a.logits = logits;
     a.dtype = dtype;

@@ -324,12 +324,8 @@ cudaError_t launch_d(const AttendArgs& a, const Plan& pl, cudaStream_t stream) {
     p.part_o = static_cast<float*>(a.workspace);
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(a.workspace) + (size_t)slots * D * sizeof(float));
     constexpr int smem = (BM + 4 * BN) * D * 2;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_mma_kernel<D>, smem); ea != cudaSuccess) return ea;
     const dim3 grid(pl.row_tiles, pl.n_splits, a.d.batch * a.d.n_kv_heads);
     attend_mma_kernel<D><<<grid, kThreads, smem, stream>>>(p);
     cudaError_t e = cudaGetLastError();

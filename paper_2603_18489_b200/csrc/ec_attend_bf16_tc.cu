@@ -506,13 +506,8 @@ cudaError_t launch_attend_bf16_tc(const AttendArgs& a, cudaStream_t stream) {
     const size_t slots = (size_t)bh * pl.n_splits * pl.rows_total;
     p.part_o = static_cast<float*>(a.workspace);
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(a.workspace) + slots * HD * sizeof(float));
-    static bool attr_done = false;
-    if (!attr_done) {
-        const cudaError_t e =
-            cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_tc_kernel, (int)SMEM_BYTES); ea != cudaSuccess) return ea;
     const dim3 grid(pl.row_tiles, pl.n_splits, bh);
     attend_tc_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(map_k, map_v, p);
     cudaError_t e = cudaGetLastError();

@@ -33,6 +33,8 @@
 #include "ec_common.cuh"
 #include "ec_tc_ptx.cuh"
 
+#include <cstdio>
+
 namespace ec {
 namespace {
 
@@ -454,6 +456,11 @@ bool attend_dense_supported(const ec_attn_desc& d, int n_active) {
     return pairs * bh >= sm_count() / 2;
 }
 
+void attend_dense_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
+    snprintf(buf, len, "attend_dense_kernel grid=(%d,%d) cluster=1", (n_active + 2 * BM - 1) / (2 * BM),
+             d.batch * d.n_q_heads);
+}
+
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     const int bh = a.d.batch * a.d.n_q_heads;
     CUtensorMap map_k, map_v;
@@ -493,14 +500,8 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
-    static bool attr_done[64] = {};   // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        const cudaError_t e = cudaFuncSetAttribute(attend_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_done[dev] = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_dense_kernel, (int)SMEM_BYTES); ea != cudaSuccess) return ea;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((p.rows_total + 2 * BM - 1) / (2 * BM), bh, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);

@@ -35,6 +35,8 @@
 #include "ec_common.cuh"
 #include "ec_tc_ptx.cuh"
 
+#include <cstdio>
+
 namespace ec {
 namespace {
 
@@ -724,15 +726,9 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
 template <int N>
 cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv,
                      const CUtensorMap& mq, int bh, cudaStream_t stream) {
-    static bool attr_done[64] = {};   // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        const cudaError_t e =
-            cudaFuncSetAttribute(attend_skip_keys_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_done[dev] = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_skip_keys_kernel<N>, (int)kSmemMax); ea != cudaSuccess)
+        return ea;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(pl.n_splits, bh, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -763,6 +759,12 @@ bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
     // row chunks re-read the K/V of a head once per chunk: only worth it while the keys can still be split
     if (pl.n_sub_r > 1 && pl.n_splits < 2) return false;
     return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && kRecvOff + kExchangeMax <= pl.off_list;
+}
+
+void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
+    const KeysPlan pl = make_keys_plan(d, n_active);
+    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u", pl.n_slots, pl.n_splits,
+             d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes);
 }
 
 cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,

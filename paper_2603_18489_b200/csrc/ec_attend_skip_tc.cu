@@ -46,6 +46,8 @@
 
 #include <cuda.h>
 
+#include <cstdio>
+
 namespace ec {
 namespace {
 
@@ -758,15 +760,8 @@ SkipPlan make_skip_plan(const ec_attn_desc& d, int n_active) {
 template <int NT>
 cudaError_t launch_nt(const SkipPlan& pl, const SkipParams& p, const CUtensorMap& mk, const CUtensorMap& mv, int bh,
                       cudaStream_t stream) {
-    static bool attr_done[64] = {};   // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        const cudaError_t e =
-            cudaFuncSetAttribute(attend_skip_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_done[dev] = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_skip_kernel<NT>, (int)kSmemMax); ea != cudaSuccess) return ea;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(pl.n_splits, bh, 1);
     cfg.blockDim = dim3(64 + NT * 128, 1, 1);
@@ -794,6 +789,12 @@ bool attend_skip_supported(const ec_attn_desc& d, int n_active) {
     const SkipPlan pl = make_skip_plan(d, n_active);
     const size_t exchange = pl.n_splits > 1 ? 2 * (size_t)pl.n_splits * pl.rows_per_cta * kRec * 4 : 0;
     return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && exchange <= pl.off_list;
+}
+
+void attend_skip_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
+    const SkipPlan pl = make_skip_plan(d, n_active);
+    snprintf(buf, len, "attend_skip_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u", pl.nt, pl.n_splits,
+             d.batch * d.n_kv_heads, pl.n_splits, pl.n_stages, pl.smem_bytes);
 }
 
 cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,

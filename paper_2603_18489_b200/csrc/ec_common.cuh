@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "entropycache.h"
 
 namespace ec {
@@ -16,7 +18,30 @@ constexpr float kLn2 = 0.6931471805599453f;
 // (B200: 148).
 constexpr int kDefaultSmCount = 148;
 
-int sm_count();  // cached cudaDevAttrMultiProcessorCount of the current device
+constexpr int kMaxDevices = 64;   // device ordinals with a slot in the per-device caches below
+
+int sm_count();  // cudaDevAttrMultiProcessorCount of the CURRENT device, cached per device ordinal
+
+// "this per-device set-up has been done" flags (cudaFuncSetAttribute is per device): one bit per ordinal, safe
+// to query and set from several host threads (a repeated set-up is harmless, a torn flag is not)
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> mask{0};
+    bool done(int dev) const { return dev >= 0 && dev < kMaxDevices && ((mask.load(std::memory_order_acquire) >> dev) & 1ull); }
+    void set(int dev) {
+        if (dev >= 0 && dev < kMaxDevices) mask.fetch_or(1ull << dev, std::memory_order_release);
+    }
+};
+
+// raises a kernel's dynamic shared-memory limit once per device
+template <typename Kernel>
+cudaError_t ensure_dynamic_smem(PerDeviceOnce& once, Kernel kernel, int bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (once.done(dev)) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) once.set(dev);
+    return e;
+}
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -57,6 +82,13 @@ struct GateArgs {
 };
 constexpr int kGateDecodeMaxRowsPerSeq = 64;
 size_t gate_workspace_bytes(int n_rows, int vocab);
+size_t gate_ticket_bytes(int n_rows);   // leading bytes of a gate workspace that must be zero when a call starts
+// all host-side argument checks of the gate entry points (EC_OK: a launch with these arguments is well-formed)
+ec_status gate_validate(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride_elems,
+                        int32_t rows_per_seq, const uint8_t* decoded_flags, uint8_t* masked, float conf_threshold,
+                        uint8_t* decoded_out, int32_t* tokens, float tau, int32_t* argmax_out, float* conf_out,
+                        float* entropy_out, float* max_entropy_out, int32_t* decision_out, float* entropy_sum_out,
+                        float* max_conf_out, const void* workspace, size_t workspace_bytes);
 cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream);
 int select_recent_max_ctx();
 cudaError_t launch_select_recent(int32_t* history, int ctx_len, int batch, ec_step_state* state, const uint8_t* decoded,
@@ -90,6 +122,11 @@ cudaError_t launch_attend_f32(const AttendArgs& a, cudaStream_t stream);
 cudaError_t launch_attend_bf16(const AttendArgs& a, cudaStream_t stream);      // mma.sync path (any head_dim)
 // fused skip-step path (bf16, head_dim 128, n_active * H_q/H_kv <= 256): refresh + attention + merge in one launch
 bool attend_skip_supported(const ec_attn_desc& d, int n_active);
+// host-only descriptions of the launch the plan functions choose ("kernel<instantiation> grid=... cluster=..."),
+// written into buf (always terminated)
+void attend_skip_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
+void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
+void attend_dense_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
 cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                cudaStream_t stream);
 // skip-step path with the keys on the M axis (bf16, head_dim 128, n_active * H_q/H_kv <= 64)

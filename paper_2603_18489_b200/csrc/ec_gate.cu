@@ -643,6 +643,8 @@ size_t gate_workspace_bytes(int n_rows, int vocab) {
     return carve(n_rows).total;
 }
 
+size_t gate_ticket_bytes(int n_rows) { return n_rows > 0 ? carve(n_rows).off_ent : 0; }   // row + sequence tickets
+
 cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     const GateWs w = carve(a.n_rows);
     char* ws = static_cast<char*>(a.workspace);

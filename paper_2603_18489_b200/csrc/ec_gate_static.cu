@@ -35,16 +35,15 @@ constexpr size_t kStaticBytes = (size_t)kStaticMaxRows * 12 + (size_t)kStaticMax
 
 static __device__ __align__(256) unsigned char g_gate_scratch[kStaticBytes];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_mu;
-void* g_scratch_addr[kMaxDevices] = {};  // device address of g_gate_scratch, per device ordinal
+void* g_scratch_addr[ec::kMaxDevices] = {};  // device address of g_gate_scratch, per device ordinal
 
 // In host code `g_gate_scratch` is only a handle for the runtime, not a device address:
 // the address a kernel can use comes from cudaGetSymbolAddress, asked once per device with
 // that device current.
 ec_status scratch_for_current_device(void** out) {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EC_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= ec::kMaxDevices) return EC_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_mu);
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
@@ -66,17 +65,20 @@ extern "C" ec_status ec_entropy_gate_static(const void* logits, int32_t dtype, i
                                             float* conf_out, float* entropy_out, float* max_entropy_out,
                                             int32_t* decision_out, void* stream) {
     if (n_rows > kStaticMaxRows) return EC_ERR_UNSUPPORTED;  // beyond the built-in scratch
-    if (n_rows <= 0 || vocab <= 0) {
-        // let the regular entry point classify the error (or accept the empty call) without scratch
-        return ec_entropy_gate(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags, tau,
-                               argmax_out, conf_out, entropy_out, max_entropy_out, decision_out, nullptr, 0, stream);
-    }
-    if (ec::gate_workspace_bytes(n_rows, vocab) > kStaticBytes) return EC_ERR_UNSUPPORTED;
+    if (n_rows > 0 && vocab > 0 && ec::gate_workspace_bytes(n_rows, vocab) > kStaticBytes) return EC_ERR_UNSUPPORTED;
+    // every argument check comes BEFORE anything is enqueued or looked up: a rejected call must leave the shared
+    // scratch alone (an earlier call's kernel may still be using it on another stream).  The checks only ask whether
+    // a workspace of kStaticBytes exists, not where it is, so they run against a placeholder address.
+    char placeholder;
+    const ec_status ok = ec::gate_validate(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags,
+                                           nullptr, 0.f, nullptr, nullptr, tau, argmax_out, conf_out, entropy_out,
+                                           max_entropy_out, decision_out, nullptr, nullptr, &placeholder, kStaticBytes);
+    if (ok != EC_OK || n_rows == 0) return ok;
     void* scratch = nullptr;
     const ec_status st = scratch_for_current_device(&scratch);
     if (st != EC_OK) return st;
     // tickets must start at zero whatever an earlier (possibly abandoned) call left behind
-    if (cudaMemsetAsync(scratch, 0, (size_t)n_rows * 8, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (cudaMemsetAsync(scratch, 0, ec::gate_ticket_bytes(n_rows), static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return EC_ERR_CUDA;
     return ec_entropy_gate(logits, dtype, n_rows, vocab, row_stride_elems, rows_per_seq, decoded_flags, tau,
                            argmax_out, conf_out, entropy_out, max_entropy_out, decision_out, scratch, kStaticBytes,

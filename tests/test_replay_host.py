@@ -74,3 +74,23 @@ def test_sliding_window_keeps_the_masked_count_constant_and_goes_non_contiguous(
     rows = st.active_rows(2)
     assert rows[:8].tolist() == win.tolist() and sorted(rows[8:].tolist()) == [p0 + 1, p0 + 4]
     assert len(set(rows.tolist())) == rows.size
+
+
+def test_harness_recent_rows_agree_with_the_oracle_on_random_histories():
+    """The harness carries its own statement of Eq. 3 (it drives both arms of the replays); here it is held against
+    the oracle's on random decode histories: ties at the threshold, fewer decoded positions than k, k = 0, dt = 0."""
+    import oracle
+    from _replay import SlidingState
+
+    rng = np.random.Generator(np.random.PCG64(2024))
+    w = syn.C1
+    for trial in range(300):
+        st = ReplayState(w) if trial % 2 == 0 else SlidingState(w, 8)
+        n_dec = int(rng.integers(0, 40))
+        pos = rng.choice(np.arange(w.prompt_len, w.ctx_len), size=n_dec, replace=False)
+        st.t = int(rng.integers(1, 12))
+        st.H[pos] = rng.integers(0, st.t + 1, size=n_dec).astype(np.float64)     # many ties
+        st.dt = int(rng.integers(0, st.t + 1))
+        k = int(rng.integers(0, 9))
+        want = oracle.select_recent(st.H, k, st.t, st.dt)
+        assert st.recent_rows(k).tolist() == want.tolist(), (trial, k, st.t, st.dt)

@@ -3,7 +3,8 @@ callers that cannot allocate device memory (a server whose HBM is already fully
 partitioned, a plug-in inside another runtime's pool).  Its scratch is a fixed
 array inside the library, shared by all calls, so this test checks that two
 calls in a row -- on different inputs, the second one smaller -- each reproduce
-what the regular entry point returns with a caller-owned workspace.  It is
+what the regular entry point returns with a caller-owned workspace, and what the
+fp64 oracle computes (Eq. 1 of the paper) within the gate's tolerances.  It is
 collected last so that a failure here cannot hide the other tests."""
 import ctypes
 
@@ -12,6 +13,7 @@ import pytest
 import torch
 
 import ec_synth as syn
+import oracle
 from _util import to_dev
 
 pytestmark = pytest.mark.gpu
@@ -49,7 +51,13 @@ def test_static_gate_matches_workspace_gate_on_two_calls_in_a_row():
         assert torch.equal(o["decision"], ref["decision"])
         for k in ("conf", "entropy", "max_entropy"):
             assert (o[k] - ref[k]).abs().max().item() <= 1e-4
-        assert float(ref["entropy"].min()) >= 0.0
+        want = oracle.entropy_gate(d["logits"], w.dtype, w.vocab, syn.decoded_flags(R, 9, rps, cfg_id=seed), tau, rps)
+        assert np.array_equal(o["argmax"].cpu().numpy(), want["argmax"])
+        assert np.abs(o["entropy"].cpu().numpy() - want["entropy"]).max() <= 1e-4
+        assert np.abs(o["conf"].cpu().numpy() - want["conf"]).max() <= 1e-5 * want["conf"].max()
+        assert np.abs(o["max_entropy"].cpu().numpy() - want["max_entropy"]).max() <= 1e-4
+        far = np.abs(want["max_entropy"] - np.float64(np.float32(tau))) >= 1e-4
+        assert np.array_equal(o["decision"].cpu().numpy()[far], want["decision"][far])
 
 
 def test_static_gate_refuses_sizes_beyond_its_scratch_and_bad_arguments():
