@@ -219,3 +219,90 @@ def test_sliding_window_replay(name, window, k):
         if abs(a["E"] - tau) >= 1e-4:
             assert a["decision"] == b["decision"]
     assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)
+
+
+@pytest.mark.parametrize("name,window,k", [("c4_llada_l2048", 32, 2), ("c4_dream_l2048", 32, 4)])
+def test_sliding_window_loop_state_kept_on_the_device(name, window, k):
+    """The paper's own decoding mode at L = 2048, both model geometries, with nothing of the loop on the host:
+    ec_entropy_gate_decode forms the decoded set and the decision, ec_select_recent_sliding updates history and mask
+    and writes the next row list, ec_attend reads that list from device memory (padded with -1 up to a fixed
+    capacity); the host reads skip_flag only.  Every step against the oracle: attention output (all real rows of a
+    partial step, sampled rows of a full one), decoded set, E, decision, history, mask, row list; at the end the
+    caches byte for byte."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.WORKLOADS[name]
+    n_steps, n_cap = 9, window + k + 8
+    dev = torch.device("cuda")
+    V = w.vocab
+
+    def step_logits(s):
+        """Window rows: Gaussian with sigma <= 3 (confidence far below 0.9), a seeded few with one logit raised by
+        about 25 (confidence practically 1), so no confidence sits near the threshold."""
+        d = syn.logits_rows(window, V, w.dtype, cfg_id=w.cfg_id, step=s, sigma_hi=3.0)
+        x = syn.decode_f64(d["logits"], w.dtype)
+        rng = np.random.Generator(np.random.PCG64(31 * s + w.cfg_id))
+        for r in rng.choice(window, size=int(rng.integers(1, 5)), replace=False):
+            x[r, int(rng.integers(0, V))] += 25.0 + 4.0 * rng.random()
+        return syn.encode(x.astype(np.float32), w.dtype)
+
+    ones = np.ones(window, np.uint8)
+    logits = [step_logits(s) for s in range(n_steps)]
+    E = sorted(float(oracle.entropy_gate_decode(lg, w.dtype, V, ones, 0.9, 0.0, window)["max_entropy"][0]) for lg in logits)
+    cut = 2 * n_steps // 3
+    assert E[cut] - E[cut - 1] > 1e-3
+    tau = float(np.float32(0.5 * (E[cut] + E[cut - 1])))          # about a third of the steps recompute
+
+    kc, vc = _caches(w)
+    okc, ovc = kc.copy(), vc.copy()
+    gk, gv = to_dev(kc), to_dev(vc)
+    d = ec.make_desc(1, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    hist, state = ec.new_history(1, w.ctx_len), ec.new_step_state(1, 1)
+    M = np.zeros(w.ctx_len, np.uint8)
+    M[w.prompt_len:] = 1
+    masked_dev = to_dev(M.copy()[None, :])
+    cur = oracle.sliding_window_rows(M, window)
+    idx_dev = torch.full((1, n_cap), -1, dtype=torch.int32, device=dev)
+    idx_dev[0, :window] = torch.from_numpy(cur.astype(np.int32)).to(dev)
+    H, t, dt, skip = np.full(w.ctx_len, -np.inf), 1, 0, False
+    rows = None
+    n_partial = 0
+    sample = sorted(np.random.Generator(np.random.PCG64(3)).choice(w.ctx_len, 10, replace=False).tolist() + [0, w.ctx_len - 1])
+    for s in range(n_steps):
+        st = state.cpu().numpy()[0]
+        assert st[0] == t and st[1] == dt and st[2] == int(skip)
+        if s == 0 or not skip:
+            tin = step_inputs(w, s, w.ctx_len)
+            out = ec.ec_attend(d, to_dev(tin["q"]), to_dev(tin["k_new"]), to_dev(tin["v_new"]), gk, gv, None, dev_status=status)
+            want = oracle.refresh_and_attend(tin["q"], tin["k_new"], tin["v_new"], okc, ovc, None, w.dtype, row_sel=sample)
+            got = to_f64(out[:, sample])
+        else:
+            n_partial += 1
+            n = rows.size
+            assert st[3] == n <= n_cap
+            tin = step_inputs(w, s, n_cap)       # the padded rows carry inputs too; their outputs are not used
+            out = ec.ec_attend(d, to_dev(tin["q"]), to_dev(tin["k_new"]), to_dev(tin["v_new"]), gk, gv, idx_dev, dev_status=status)
+            want = oracle.refresh_and_attend(tin["q"][:, :n], tin["k_new"][:, :n], tin["v_new"][:, :n], okc, ovc,
+                                             rows[None, :].astype(np.int32), w.dtype)
+            got = to_f64(out)[:, :n]
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.abs(want - got).max() <= 1e-2, s
+        o = oracle.entropy_gate_decode(logits[s], w.dtype, V, ones, 0.9, tau, window)
+        assert not (np.abs(o["conf"] - np.float64(np.float32(0.9))) <= 1e-3).any()
+        tok = torch.full((window,), -1, dtype=torch.int32, device=dev)
+        g = ec.ec_entropy_gate_decode(to_dev(logits[s]), V, window, to_dev(ones.copy()), 0.9, tau, tok)
+        assert np.array_equal(g["decoded"].cpu().numpy(), o["decoded"]), s
+        assert abs(float(g["max_entropy"][0]) - o["max_entropy"][0]) <= 1e-4 and abs(o["max_entropy"][0] - tau) >= 1e-4
+        assert int(g["decision"][0]) == int(o["decision"][0])
+        ec.ec_select_recent_sliding(hist, state, masked_dev, g["decoded"], window, g["decision"], k, idx_dev)
+        new_rows, skip, dt, t = oracle.sliding_step_bookkeeping(H, M, t, dt, cur, o["decoded"], int(o["decision"][0]), k, window)
+        cur = new_rows[:min(window, int(M.sum()))]
+        rows = new_rows
+        assert np.array_equal(hist.cpu().numpy()[0].astype(np.int64), np.where(np.isfinite(H), H, -(2 ** 31)).astype(np.int64))
+        assert np.array_equal(masked_dev.cpu().numpy()[0], M)
+        g_idx = idx_dev.cpu().numpy()[0]
+        assert g_idx[:rows.size].tolist() == rows.tolist() and np.all(g_idx[rows.size:] == -1)
+    assert n_partial >= 3
+    assert np.array_equal(to_storage(gk), okc) and np.array_equal(to_storage(gv), ovc)
