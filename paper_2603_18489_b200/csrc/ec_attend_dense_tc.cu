@@ -59,32 +59,6 @@ constexpr uint32_t TM_S = 0, TM_O = 256;   // + 128 * tile
 enum { B_FULL = 0, B_EMPTY = kSlots, B_SFULL = 2 * kSlots, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_COUNT = B_QFULL + 1 };
 
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pk(float lo, float hi) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void upk(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
-    f32x2 r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
-__device__ __forceinline__ void named_barrier(int id, int n_threads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
 // 2^x for a pair of values on the FMA pipe (the MUFU pipe is the softmax's bottleneck, so a share of the
 // exponentials is computed here instead): x = n + f with n = round(x), |f| <= 1/2, 2^f by a cubic fitted for a
 // maximum relative error of 7.5e-5 (far below the bf16 rounding of P), and n added to the exponent field.
@@ -409,23 +383,6 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 // ---- host side ---------------------------------------------------------------------------
 // Q of an MHA step seen as 5-D {64 columns, active row, head, half, sequence}: one box {64, 128, 1, 2, 1} lands as the
 // two 128-byte-swizzled halves of a [128 rows x 128] tile; rows past n_active read as zero.
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
 // K or V seen as 5-D {64 columns, key, half, kv head, sequence}: one box {64, 128, 2, 1, 1} lands as
 // [half][key][64 columns], the two 128-byte-swizzled halves of a [128 keys x 128] tile; keys beyond L read as zero.
 // Cache layout [B, Hkv, L, 128] or token-major [B, L, Hkv, 128] (the fresh K/V of a recompute step): only the

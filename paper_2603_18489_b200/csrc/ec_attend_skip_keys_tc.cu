@@ -1,37 +1,44 @@
-// ec_attend, skip step with FEW query rows (bf16, head_dim 128, at most 64 packed query rows per kv head):
+// ec_attend, skip step with FEW query rows (bf16, head_dim 128, at most 96 packed query rows per CTA column):
 // ONE launch that refreshes the active rows' K/V in the cache, attends from the active rows over the whole
 // cache and merges the key-range partials.  (Section 4.2 and Appendix A of the paper, partial branch:
 // TransformerBlock(Q[M u R], K[I], V[I]) after the rows M u R got fresh K, V.)
 //
 // With 34 query rows a 128-row M tile would be three quarters padding, and a thread per query row would
 // leave most softmax lanes idle.  Here the KEYS take the M axis of the tensor core and the query rows the N
-// axis (N = 48 or 64):
+// axis (N = 48, 64 or 96 slots):
 //     S^T[128 keys x N]  = K_tile[128 keys x 128] . Q[N x 128]^T          (A = K tile, B = Q, both K-major)
 //     O^T[128 d    x N] += V_tile^T[128 d x 128 keys] . P^T[128 keys x N]  (A = V tile MN-major, B = P^T MN-major)
-// so a softmax thread owns one KEY (TMEM lane) and N scores: all 128 softmax lanes work, one exponential per
-// (key, query) and no padding rows, and a step of the pipeline covers 128 keys.
+//     L^T[128      x N] += 1[128 x 128 keys]          . P^T[128 keys x N]  (A = a block of ones in tensor memory)
+// so a softmax thread owns one KEY (TMEM lane) and its scores against the query slots: all 128 lanes work, one
+// exponential per (key, query), no padding rows, a pipeline step covers 128 keys.  The row sums come out of the
+// tensor core as well (every lane of L^T holds sum_keys P), so the softmax threads carry no running sums and
+// nothing has to be reduced across threads at the end.  With N = 96 (the paper's default budget k = 64 gives 96
+// active rows) two softmax warpgroups share the columns of a key.
 //   softmax  the reference maxima m[q] (log2 units) are shared by all keys of the CTA and live in shared memory.
 //            The common path computes p = 2^(s*scale*log2e - m[q]) with no reduction at all; a barrier-wide OR
 //            tells whether any score exceeds its reference by more than 2^8 (always true on the first tile):
-//            only then the column maxima are reduced (integer warp reductions + shared memory), m is raised,
-//            and O^T and the partial row sums are rescaled.  Row sums are kept per thread (sum over its own
-//            keys) and reduced across the CTA once, at the end;
-//   grid     (C, B*H_kv*n_sub) as clusters of C in {1, 2, 4, 8} CTAs that split one head's 128-key tiles.  With
-//            grouped-query attention the g = H_q/H_kv query heads of a kv head are packed into the N axis; when
-//            n*g exceeds the 64 slots the heads are spread over n_sub CTA columns (each takes g/n_sub heads and
-//            streams the same K/V, which the other columns' reads keep in L2).  Every column refreshes the rows of
-//            its key range itself: the columns of a kv head write identical bytes, and each orders its own copy
-//            before its own TMA reads, so whichever copy a read observes holds the fresh row;
-//   refresh  as in the row-major skip kernel: a CTA refreshes the cache rows of its own key range, visits its
-//            tiles in rotated order and waits for the copy only before the first tile that holds one;
-//   merge    CTA c of the cluster owns the output columns d in [c*128/C, (c+1)*128/C): every CTA sends that
-//            slice of its O^T (rows of the TMEM accumulator) plus its m and l vectors with one bulk
-//            shared-to-shared copy per owner; the owner combines, normalises and writes out[b, i, h, d].
-// warp 0: TMA producer (K and V tiles of 128 keys, one 4-D box each, NS stages of 64 KB); warp 1: refresh list
-// and tcgen05.mma issue; warps 2..5: Q staging, refresh copy, softmax, exchange.  One CTA per SM.
-// Launched with programmatic stream serialisation; global memory is touched only after griddepcontrol.wait.
-// Every mbarrier wait is bounded (EC_ERR_TIMEOUT in dev_status, CTA-wide abort flag); the CTA always frees its
-// TMEM and exits.
+//            only then the column maxima are reduced, m is raised, and O^T and L^T are rescaled;
+//   grid     (C, B*H_kv*n_sub) as clusters of C <= 8 CTAs (any count, not only powers of two) that split one
+//            head's 128-key tiles, chosen so that the most-loaded SM streams the fewest tiles; CTAs that hold a
+//            single tile are small enough for two per SM.  With grouped-query attention the query heads of a kv
+//            head are packed into the N axis; when they exceed the slots the heads (and, beyond 96 active rows,
+//            the rows) are spread over n_sub CTA columns that stream the same K/V (L2 serves the repeats);
+//   K/V      the producer warp issues its TMA loads at once, in key order, through a ring of NS stages of 64 KB:
+//            they depend on nothing;
+//   refresh  the active rows' fresh K/V reach the attention through SHARED memory, not through the cache: two
+//            patch warps copy the fresh rows of the CTA's key range from k_new / v_new over the stale rows of the
+//            landed tile (same swizzled layout the TMA wrote) before that tile's first product is issued, and
+//            write the same bytes into the cache in global memory for later steps.  Whether a concurrent TMA
+//            read of such a row saw the old or the new bytes does not matter, so nothing orders the cache update
+//            against the loads;
+//   merge    CTA c of the cluster owns the output columns d in [c*DL, (c+1)*DL): once every CTA of the cluster is
+//            past its main loop (first cluster barrier) each softmax thread stores its O^T row (one output column,
+//            all queries) straight into the owner's shared memory, plus m and l; after the second cluster barrier
+//            the owner combines the C partials, normalises and writes out[b, i, h, d].
+// warp 0: TMA producer; warp 1: refresh list, then tcgen05.mma issue; next 4 (or 8) warps: softmax; last two
+// warps: patch / refresh.  Launched with programmatic stream serialisation; global memory is touched only after
+// griddepcontrol.wait.  Every mbarrier wait is bounded (EC_ERR_TIMEOUT in dev_status, CTA-wide abort flag: an
+// aborted CTA stores no output); the CTA always frees its TMEM and exits.
 #include "ec_common.cuh"
 #include "ec_tc_ptx.cuh"
 
@@ -43,58 +50,54 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 128, HD = 128;
-constexpr int kThreads = 192;
-constexpr int kSoft = 128;
+constexpr int kAuxThreads = 64;           // two warps: refresh patches and row sums
+constexpr int kPatchPer = 18;             // 16-byte pieces of fresh rows a thread holds per round (36 rows per round)
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr uint32_t STAGE = 2 * TILE;       // K tile + V tile: 64 KB
-constexpr uint32_t P_BYTES = SUB;          // P^T [128 keys x 64 query slots] bf16
 constexpr int kMaxStages = 3;
-constexpr int kMaxRowsT = 64;            // query slots (packed rows) of one CTA
-constexpr int kMaxActive = 256;          // active rows of a sequence (refresh list, row chunks)
-constexpr uint32_t TM_COLS = 256;          // S^T buffers at columns 0 and 64, O^T at 128
-constexpr uint32_t TM_S = 0, TM_O = 128;
-// exchange areas, reusing the dead staging memory after the main loop (bytes from the aligned base)
-constexpr uint32_t kStagingOff = 36864;                       // row-sum scratch [128][N + 1] floats sits below it
-constexpr uint32_t kExchangeMax = (128 * 65 + 2 * 64 * 8) * 4;   // C chunks of (128/C) x (N + 1) + 2N floats, N <= 64, C <= 8
-constexpr uint32_t kRecvOff = kStagingOff + 40960;
+constexpr int kMaxSlots = 96;              // query slots (packed rows) of one CTA column
+constexpr int kMaxActive = 256;            // active rows of a sequence (refresh list, row chunks)
+constexpr int kMaxTiles = 1024;            // key tiles of one CTA (bits of the patch mask)
 
 enum { B_FULL = 0, B_EMPTY = kMaxStages, B_SFULL = 2 * kMaxStages, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 1,
-       B_QFULL = B_PVDONE + 1, B_LIST = B_QFULL + 1, B_REFRESHED = B_LIST + 1, B_RECV = B_REFRESHED + 1, B_COUNT = B_RECV + 1 };
+       B_PSUM = B_PVDONE + 1, B_QFULL = B_PSUM + 1, B_LIST = B_QFULL + 1, B_NEEDPATCH = B_LIST + 1,
+       B_PATCHED = B_NEEDPATCH + kMaxStages, B_RECV = B_PATCHED + kMaxStages, B_COUNT = B_RECV + 1 };
 
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pk(float lo, float hi) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void upk(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
-    f32x2 r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
-    f32x2 r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
+constexpr uint32_t kBarBytes = (B_COUNT * 8u + 15u) & ~15u;   // the barrier block, padded so that what follows is 16-byte aligned
+
 // order-preserving map float -> int (for integer warp reductions of a maximum) and back
 __device__ __forceinline__ int f2ord(float f) {
     const int i = __float_as_int(f);
     return i >= 0 ? i : (i ^ 0x7fffffff);
 }
 __device__ __forceinline__ float ord2f(int i) { return __int_as_float(i >= 0 ? i : (i ^ 0x7fffffff)); }
+
+// COLS consecutive 32-bit columns of this thread's TMEM lane -> registers (and back).  ALIGNED32: the first column is
+// a multiple of 32 (one 32-column access, then the rest); otherwise 16-column accesses at multiples of 16.
+template <int COLS, bool ALIGNED32>
+__device__ __forceinline__ void ld_row(uint32_t taddr, uint32_t* r) {
+    static_assert(COLS == 48 || COLS == 64, "columns per thread");
+    if (ALIGNED32) {
+        ld32(taddr, r);
+        if (COLS == 48) ld16(taddr + 32, r + 32); else ld32(taddr + 32, r + 32);
+    } else {
+#pragma unroll
+        for (int c = 0; c < COLS; c += 16) ld16(taddr + c, r + c);
+    }
+    wait_ld();
+}
+template <int COLS, bool ALIGNED32>
+__device__ __forceinline__ void st_row(uint32_t taddr, const uint32_t* r) {
+    if (ALIGNED32) {
+        st32(taddr, r);
+        if (COLS == 48) st16(taddr + 32, r + 32); else st32(taddr + 32, r + 32);
+    } else {
+#pragma unroll
+        for (int c = 0; c < COLS; c += 16) st16(taddr + c, r + c);
+    }
+    wait_st();
+}
 
 struct KeysParams {
     const __nv_bfloat16* q;
@@ -111,7 +114,8 @@ struct KeysParams {
     int n_sub_r;      // row chunks = ceil(n_active / rows_chunk)
     int n_sub;        // CTA columns per kv head = ((H_q / H_kv) / group) * n_sub_r
     int n_splits, tiles_per_split, n_stages;
-    int q_tma;                    // 1: the producer fetches Q with one TMA box (MHA); 0: the softmax warps stage it
+    int dl;           // output columns merged by one CTA of the cluster (even; the last CTA may own fewer)
+    int q_tma;        // 1: the producer fetches Q with one TMA box (one query head per column); 0: softmax warps stage it
     uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0
     float scale_log2;
 };
@@ -120,25 +124,36 @@ struct KeysParams {
 struct alignas(16) KeysShared {
     uint32_t tmem;
     int abort_flag;
-    int n_mine;       // entries of the refresh list
-    int spec_ok;      // 1: the first tile of the range, loaded before the list was known, holds no refreshed row
-    int first_tile;   // rotation of the visiting order, see tile_of()
-    int j_refreshed;  // first visit index j whose tile holds a refreshed position (T if none)
-    alignas(16) float m[kMaxRowsT];        // reference maxima of the query rows, log2 units (read as float2)
-    alignas(16) float factor[kMaxRowsT];   // rescale factors of the current slow path; the row sums at the end
-    int colmax[4][kMaxRowsT];      // per-warp column maxima (ordered ints) of the current slow path
+    int n_mine;                                // entries of the refresh list
+    int pad;
+    int slow_flag[2][2];                       // [tile parity][warpgroup]: the softmax of that tile raised its references
+    uint32_t patch_mask[kMaxTiles / 32];       // bit j: tile j of this CTA holds a refreshed position
+    alignas(16) float m[kMaxSlots];            // reference maxima of the query rows, log2 units (read as float2)
+    alignas(16) float factor[2][kMaxSlots];    // [tile parity]: rescale factors of that tile's slow path
+    alignas(16) float lpart[2][kMaxSlots];     // row sums of the CTA's keys, one partial per group of row-sum threads
+    int colmax[4][kMaxSlots];                  // per-warp column maxima (ordered ints) of the current slow path
 };
 
 template <int N>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(64 + (N > 64 ? 256 : 128) + kAuxThreads, N <= 64 ? 2 : 1)
 attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_q, const KeysParams p) {
-    static_assert(N == 48 || N == 64, "query-row slots per CTA");
+    static_assert(N == 48 || N == 64 || N == 96, "query-row slots per CTA");
+    constexpr int WG = N > 64 ? 2 : 1;          // softmax warpgroups: each takes NH of a key's N scores
+    constexpr int NH = N / WG;
+    constexpr int kSoft = 128 * WG;
+    constexpr int kThreads = 64 + kSoft + kAuxThreads;
+    // tensor-memory columns: S^T x 2 and O^T at multiples of NP (the slots rounded up to 64 or 128)
+    constexpr uint32_t NP = N <= 64 ? 64 : 128;
+    constexpr uint32_t TM_S = 0, TM_O = 2 * NP;
+    constexpr uint32_t TM_COLS = (3 * NP <= 256) ? 256 : 512;
+    // row-sum threads: a column pair and a share of the tile's keys each
+    constexpr int kPairs = N / 2, kParts = (kAuxThreads / kPairs) >= 2 ? 2 : 1;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (s2u(smem_raw) + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - s2u(smem_raw));
     const uint32_t bars = base + p.off_bar;
-    KeysShared* sh = reinterpret_cast<KeysShared*>(gbase + p.off_bar + B_COUNT * 8);
+    KeysShared* sh = reinterpret_cast<KeysShared*>(gbase + p.off_bar + kBarBytes);
     volatile int* abort_flag = &sh->abort_flag;
     int2* list = reinterpret_cast<int2*>(gbase + p.off_list);   // (active row i, position) pairs of this CTA's key range
     auto bar = [&](int idx) { return bars + idx * 8; };
@@ -150,15 +165,21 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int i0 = (sub % p.n_sub_r) * p.rows_chunk;                           // first active row of this CTA
     const int rows_total = min(p.rows_chunk, p.n_active - i0) * p.group;       // packed query rows of this CTA
     const int C = p.n_splits;
-    const int DL = HD / C;                                 // output columns this CTA merges
+    const int DL = p.dl;
     const int n_tiles_total = (p.ctx_len + BK - 1) / BK;
     const int t_begin = split * p.tiles_per_split;
     const int t_end = min(n_tiles_total, t_begin + p.tiles_per_split);
     const int T = t_end - t_begin;   // >= 1 by construction of the plan
     const int NS = p.n_stages;
     const bool refresh = p.k_new != nullptr;
-    constexpr int NP = N + 1;   // odd row stride (floats) of the transposing buffers: conflict-free by row and by column
-    const uint32_t chunk_bytes = (uint32_t)(DL * NP + 2 * N) * 4u;   // one owner's slice of O^T, then m[N], l[N]
+    const int key_lo = t_begin * BK, key_hi = min(p.ctx_len, t_end * BK);
+    // exchange areas of the merge, from the start of the (then dead) Q / P^T / stage memory: C staging chunks (one per
+    // owner), C receive chunks (one per source), the weight table, the rows' output offsets.  A chunk holds
+    // [N queries][DL columns] floats of O^T, then m[N], then l[N].
+    const uint32_t chunk_floats = (uint32_t)(N * DL + 2 * N);
+    const uint32_t chunk_bytes = chunk_floats * 4u;
+    const uint32_t stg_off = 0, recv_off = (uint32_t)C * chunk_bytes, wgt_off = 2u * C * chunk_bytes,
+                   qoff_off = wgt_off + 8u * N * 4u;
 
     // ---- set-up (touches no global memory) -------------------------------------------------
     if (tid == 0) {
@@ -167,17 +188,16 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (p.q_tma) prefetch_map(&map_q);
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1;
-            if (i == B_PFULL || i == B_REFRESHED || (i == B_QFULL && !p.q_tma)) count = kSoft;
+            if (i == B_PFULL || (i == B_QFULL && !p.q_tma)) count = kSoft;
+            if (i == B_PSUM || (i >= B_PATCHED && i < B_PATCHED + kMaxStages)) count = kAuxThreads;
             mbar_init(bar(i), count);
         }
         sh->abort_flag = 0;
         sh->n_mine = 0;
-        sh->spec_ok = 1;
-        sh->first_tile = 0;
-        sh->j_refreshed = T;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (C > 1) mbar_expect_tx(bar(B_RECV), (uint32_t)C * chunk_bytes);
+        if (C > 1) mbar_expect_tx(bar(B_RECV), (uint32_t)C * chunk_bytes);   // the peers' partials, one chunk each
     }
+    if (tid < kMaxTiles / 32) sh->patch_mask[tid] = 0u;
     if (tid < N) sh->m[tid] = -INFINITY;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(&sh->tmem)), "r"(TM_COLS)
@@ -191,16 +211,6 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     pdl_wait();                    // the previous kernel of the stream has completed; global memory may be touched
     pdl_launch_dependents();
 
-    const int key_lo = t_begin * BK, key_hi = min(p.ctx_len, t_end * BK);
-    // Visiting order of the CTA's T tiles.  The producer loads the first tile of the range at once, before the
-    // refresh list is known.  If that tile holds no refreshed row (spec_ok) it is visit 0 and the other tiles
-    // follow in rotated order, those without refreshed rows first; otherwise its data are discarded (that stage
-    // is simply filled again later) and all T tiles are visited in rotated order, shifted by one stage.
-    auto tile_of = [&](int j, int spec_ok, int rot) {
-        if (spec_ok) return j == 0 ? 0 : 1 + (rot + j - 1) % (T - 1);
-        return (rot + j) % T;
-    };
-
     if (warp == 0) {
         // ================================ TMA producer ======================================
         if (lane == 0) {
@@ -208,50 +218,18 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
                 tma_load_5d(base, &map_q, 0, i0, hq0, 0, b, bar(B_QFULL));   // rows past the chunk land in unused slots
             }
-            auto load_tile = [&](int tile, int stage) {
-                const int key0 = (t_begin + tile) * BK;
-                const uint32_t dst = base + p.off_stage + stage * STAGE;
-                mbar_expect_tx(bar(B_FULL + stage), STAGE);
-                tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + stage));
-                tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + stage));
-            };
-            int spec_ok = 1, rot = 0, j_refreshed = T;
-            load_tile(0, 0);   // visit 0 if it turns out to hold no refreshed row
-            if (refresh) {
-                mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
-                spec_ok = sh->spec_ok;
-                rot = sh->first_tile;
-                j_refreshed = sh->j_refreshed;
+            for (int j = 0; j < T; ++j) {
+                const int s = j % NS, u = j / NS;
+                if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
+                const int key0 = (t_begin + j) * BK;
+                const uint32_t dst = base + p.off_stage + s * STAGE;
+                mbar_expect_tx(bar(B_FULL + s), STAGE);
+                tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
+                tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
             }
-            const int soff = spec_ok ? 0 : 1;   // stage shift: the discarded fill took stage 0's first phase
-            bool discard_seen = spec_ok != 0;
-            for (int j = spec_ok ? 1 : 0; j < T; ++j) {
-                const int s = (j + soff) % NS, u = (j + soff) / NS;
-                if (j == j_refreshed) mbar_wait(bar(B_REFRESHED), 0, abort_flag, p.dev_status);
-                if (u > 0) {
-                    if (soff == 1 && s == 0) {
-                        // stage 0: its phase 0 was the discarded fill, which nobody consumes or releases
-                        if (u == 1) {
-                            mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);
-                            discard_seen = true;
-                        } else {
-                            mbar_wait(bar(B_EMPTY + 0), (u - 2) & 1, abort_flag, p.dev_status);
-                        }
-                    } else {
-                        mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
-                    }
-                }
-                load_tile(tile_of(j, spec_ok, rot), s);
-            }
-            if (!discard_seen) mbar_wait(bar(B_FULL + 0), 0, abort_flag, p.dev_status);   // no copy in flight at exit
-        }
-        if (C > 1) {   // this warp no longer touches the memory the peers' partials will land in
-            __syncwarp();
-            cluster_arrive();
         }
     } else if (warp == 1) {
         // ================= refresh list, then MMA issue (lane 0) =================================
-        bool spec_ok_w1 = true;
         if (refresh) {
             int posv[kMaxActive / 32];
 #pragma unroll
@@ -261,7 +239,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 if (k * 32 >= p.n_active) continue;   // uniform: nothing of the list left
                 if (i < p.n_active) posv[k] = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
             }
-            int n_mine = 0, hi_tile = -1, lo_tile = T;   // last / first local tile that holds a refreshed position
+            int n_mine = 0;
 #pragma unroll
             for (int k = 0; k < kMaxActive / 32; ++k) {
                 if (k * 32 >= p.n_active) break;
@@ -269,72 +247,49 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 const unsigned mk = __ballot_sync(0xffffffffu, hit);
                 if (hit) {
                     list[n_mine + __popc(mk & ((1u << lane) - 1u))] = make_int2(k * 32 + lane, posv[k]);
-                    hi_tile = max(hi_tile, (posv[k] - key_lo) / BK);
-                    lo_tile = min(lo_tile, (posv[k] - key_lo) / BK);
+                    const int tile = (posv[k] - key_lo) / BK;
+                    atomicOr(&sh->patch_mask[tile >> 5], 1u << (tile & 31));
                 }
                 n_mine += __popc(mk);
             }
-            hi_tile = __reduce_max_sync(0xffffffffu, hi_tile);
-            lo_tile = __reduce_min_sync(0xffffffffu, lo_tile);
-            spec_ok_w1 = lo_tile > 0;   // the tile loaded ahead of this list holds no refreshed row
-            int rot = 0;
-            if (n_mine > 0) rot = spec_ok_w1 ? hi_tile % (T - 1) : (hi_tile + 1) % T;   // (spec_ok and n_mine > 0 imply T > 1)
-            int j_ref = T;
-#pragma unroll
-            for (int k = 0; k < kMaxActive / 32; ++k) {
-                if (k * 32 >= p.n_active) break;
-                if (posv[k] >= key_lo && posv[k] < key_hi) {
-                    const int tile = (posv[k] - key_lo) / BK;
-                    int j;
-                    if (spec_ok_w1) {
-                        j = tile - 1 - rot;
-                        if (j < 0) j += T - 1;
-                        j += 1;
-                    } else {
-                        j = tile - rot;
-                        if (j < 0) j += T;
-                    }
-                    j_ref = min(j_ref, j);
-                }
-            }
-            j_ref = __reduce_min_sync(0xffffffffu, j_ref);
             __syncwarp();
             if (lane == 0) {
                 sh->n_mine = n_mine;
-                sh->spec_ok = spec_ok_w1 ? 1 : 0;
-                sh->first_tile = rot;
-                sh->j_refreshed = j_ref;
-                mbar_arrive(bar(B_LIST));
+                mbar_arrive(bar(B_LIST));   // release: the list and the mask above are visible to whoever waits
             }
+            __syncwarp();
         }
         if (lane == 0) {
             constexpr uint32_t IDESC_S = instr_desc2(N, 0, 0);    // A = K tile (K-major), B = Q (K-major)
             constexpr uint32_t IDESC_PV = instr_desc2(N, 1, 1);   // A = V tile (MN-major: d contiguous), B = P^T (MN-major)
             constexpr uint32_t QHALF = N * 128;                   // bytes of one 64-column half of the Q tile
-            const int soff = spec_ok_w1 ? 0 : 1;
-            auto stage_of = [&](int j) { return (j + soff) % NS; };
-            auto wait_stage = [&](int j) { mbar_wait(bar(B_FULL + stage_of(j)), ((j + soff) / NS) & 1, abort_flag, p.dev_status); };
+            // A tile that holds refreshed positions is handed to the patch warps once it has landed ("needs patch")
+            // and used once they are done ("patched"); one barrier pair per stage, and this thread waits for the
+            // answer before it goes on, so neither side can run a phase ahead of the other.
+            uint32_t n_patched = 0;   // bit s: parity of the patches of stage s so far
             auto issue_s = [&](int j) {
-                const uint32_t kst = base + p.off_stage + stage_of(j) * STAGE;
+                const int s = j % NS;
+                mbar_wait(bar(B_FULL + s), (j / NS) & 1, abort_flag, p.dev_status);
+                if (refresh && ((sh->patch_mask[j >> 5] >> (j & 31)) & 1u)) {
+                    mbar_arrive(bar(B_NEEDPATCH + s));
+                    mbar_wait(bar(B_PATCHED + s), (n_patched >> s) & 1u, abort_flag, p.dev_status);
+                    n_patched ^= 1u << s;
+                }
+                fence_after();
+                const uint32_t kst = base + p.off_stage + s * STAGE;
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t koff = (k & 3) * 32;
-                    mma_ss(tmem + TM_S + (j & 1) * 64, smem_desc(kst + (k >> 2) * SUB + koff, 16, 1024),
+                    mma_ss(tmem + TM_S + (j & 1) * NP, smem_desc(kst + (k >> 2) * SUB + koff, 16, 1024),
                            smem_desc(base + (k >> 2) * QHALF + koff, 16, 1024), IDESC_S, k > 0);
                 }
                 commit(bar(B_SFULL + (j & 1)));
             };
             mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
-            wait_stage(0);
-            fence_after();
             issue_s(0);
             for (int j = 0; j < T; ++j) {
-                if (j + 1 < T) {
-                    wait_stage(j + 1);
-                    fence_after();
-                    issue_s(j + 1);
-                }
-                const uint32_t vst = base + p.off_stage + stage_of(j) * STAGE + TILE;
+                if (j + 1 < T) issue_s(j + 1);
+                const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + TILE;
                 mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
                 fence_after();
 #pragma unroll
@@ -342,16 +297,118 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                     mma_ss(tmem + TM_O, smem_desc(vst + k * 2048, SUB, 1024), smem_desc(base + p.off_p + k * 2048, SUB, 1024),
                            IDESC_PV, (j > 0 || k > 0));
                 commit(bar(B_PVDONE));
-                commit(bar(B_EMPTY + stage_of(j)));
+                commit(bar(B_EMPTY + j % NS));
             }
         }
-        if (C > 1) {   // (the products still in flight are covered by the softmax warps, which arrive after the last one)
-            __syncwarp();
-            cluster_arrive();
+    } else if (warp >= 2 + 4 * WG) {
+        // ===== auxiliary warps: fresh rows over the landed tiles (and into the cache); row sums of P^T =====
+        const int atid = tid - (64 + kSoft);
+        int n_mine = 0;
+        if (refresh) {
+            mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
+            n_mine = sh->n_mine;
+        }
+        const bool writer = sub == 0;   // one CTA column per kv head updates the cache in global memory
+        // 16-byte pieces of the list's rows that fall into tile j: entry e = c >> 5, K pieces 0..15 then V pieces 0..15.
+        // A thread holds up to kPatchPer pieces of one round in registers, so the loads of a tile's fresh rows are in
+        // flight while the tile itself is still landing.
+        uint4 pv[kPatchPer];
+        auto patch_loads = [&](int j, int round) {
+            const int key0 = key_lo + j * BK;
+#pragma unroll
+            for (int u = 0; u < kPatchPer; ++u) {
+                const int c = (round * kPatchPer + u) * kAuxThreads + atid;
+                if (c < n_mine * 32) {
+                    const int2 ip = list[c >> 5];
+                    if (ip.y >= key0 && ip.y < key0 + BK) {
+                        const long long src = (((long long)b * p.n_active + ip.x) * p.n_kv_heads + hk) * HD + (c & 15) * 8;
+                        pv[u] = __ldg(reinterpret_cast<const uint4*>(((c & 16) ? p.v_new : p.k_new) + src));
+                    }
+                }
+            }
+        };
+        auto patch_stores = [&](int j, int round) {
+            const int key0 = key_lo + j * BK;
+            unsigned char* kt = gbase + p.off_stage + (j % NS) * STAGE;
+#pragma unroll
+            for (int u = 0; u < kPatchPer; ++u) {
+                const int c = (round * kPatchPer + u) * kAuxThreads + atid;
+                if (c < n_mine * 32) {
+                    const int2 ip = list[c >> 5];
+                    if (ip.y >= key0 && ip.y < key0 + BK) {
+                        const int r = ip.y - key0, piece = c & 15, isv = (c >> 4) & 1;
+                        const uint32_t off = (uint32_t)isv * TILE + (uint32_t)(piece >> 3) * SUB + (r >> 3) * 1024 + (r & 7) * 128 +
+                                             (((piece & 7) ^ (r & 7)) << 4);
+                        *reinterpret_cast<uint4*>(kt + off) = pv[u];
+                        if (writer)
+                            *reinterpret_cast<uint4*>((isv ? p.v_cache : p.k_cache) + ((long long)bh * p.ctx_len + ip.y) * HD + piece * 8) =
+                                pv[u];
+                    }
+                }
+            }
+        };
+        auto next_patched = [&](int from) {   // first tile >= from that holds a refreshed position (T if none)
+            for (int j = from; j < T; ++j)
+                if ((sh->patch_mask[j >> 5] >> (j & 31)) & 1u) return j;
+            return T;
+        };
+        const int n_rounds = (n_mine * 32 + kPatchPer * kAuxThreads - 1) / (kPatchPer * kAuxThreads);
+        int np = n_mine > 0 ? next_patched(0) : T;
+        if (np < T) patch_loads(np, 0);
+        uint32_t n_needed = 0;   // bit s: parity of the "needs patch" hand-overs of stage s so far
+
+        // row sums: this thread adds up column pair cp of the keys [k_lo, k_lo + BK / kParts) of every tile
+        const bool summer = atid < kPairs * kParts;
+        const int cp = atid % kPairs, col = 2 * cp, gch = col >> 3;
+        const int k_lo = (atid / kPairs) * (BK / kParts);
+        const unsigned char* pcol = gbase + p.off_p + (gch >> 3) * SUB + (col & 7) * 2;
+        float acc0 = 0.f, acc1 = 0.f;
+
+        for (int j = 0; j < T; ++j) {
+            // every tile up to j + 1 that needs its fresh rows gets them now: S of tile j + 1 is issued before P V of tile j
+            while (np <= j + 1 && np < T) {
+                const int s = np % NS;
+                mbar_wait(bar(B_NEEDPATCH + s), (n_needed >> s) & 1u, abort_flag, p.dev_status);   // the tile has landed
+                n_needed ^= 1u << s;
+                for (int round = 0; round < n_rounds; ++round) {
+                    if (round > 0) patch_loads(np, round);
+                    patch_stores(np, round);
+                }
+                fence_async_smem();     // patched rows (generic proxy) -> visible to the tensor core (async proxy)
+                mbar_arrive(bar(B_PATCHED + s));
+                np = next_patched(np + 1);
+                if (np < T) patch_loads(np, 0);
+            }
+            // P^T of tile j is in shared memory
+            mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
+            if (summer) {
+                if (sh->slow_flag[j & 1][col / NH]) {   // the references of these columns were raised at this tile
+                    acc0 *= sh->factor[j & 1][col];
+                    acc1 *= sh->factor[j & 1][col + 1];
+                }
+#pragma unroll 4
+                for (int k8 = 0; k8 < BK / kParts; k8 += 8) {
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const int k = k_lo + k8 + r;
+                        const uint32_t w = *reinterpret_cast<const uint32_t*>(pcol + (k >> 3) * 1024 + r * 128 + (((gch & 7) ^ r) << 4));
+                        acc0 += __uint_as_float(w << 16);
+                        acc1 += __uint_as_float(w & 0xffff0000u);
+                    }
+                }
+                if (j == T - 1) {
+                    sh->lpart[atid / kPairs][col] = acc0;
+                    sh->lpart[atid / kPairs][col + 1] = acc1;
+                }
+            }
+            mbar_arrive(bar(B_PSUM));   // P^T of tile j has been read (release: the row sums above are visible)
         }
     } else {
-        // ================== Q staging, cache refresh, softmax (warps 2..5) ========================
+        // ================== Q staging (grouped heads), softmax (warps 2 ..) ========================
         const int stid = tid - 64;
+        const int wg = stid >> 7;                    // warpgroup: columns [wg * NH, (wg + 1) * NH) of every key
+        const int c0 = wg * NH;
+        const int st_w = stid & 127;
         constexpr uint32_t QHALF = N * 128;
         // Q rows of this kv head -> swizzled K-major tile of N rows (rows past rows_total are zero)
         for (int c = stid; c < (p.q_tma ? 0 : N * (HD / 8)); c += kSoft) {
@@ -370,131 +427,94 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             mbar_arrive(bar(B_QFULL));
         }
 
-        int spec_ok = 1, rot = 0;
-        if (refresh) {
-            mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
-            spec_ok = sh->spec_ok;
-            rot = sh->first_tile;
-            // fresh rows of this CTA's key range -> cache in global memory, eight 16-byte pieces in flight per thread
-            const int chunks = sh->n_mine * 32;
-            for (int c0 = stid; c0 < chunks; c0 += 8 * kSoft) {
-                uint4 v[8];
-                long long dsto[8];
-                int isv[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = c0 + u * kSoft;
-                    isv[u] = -1;
-                    if (c < chunks) {
-                        const int e = c >> 5, piece = c & 15;
-                        isv[u] = (c >> 4) & 1;
-                        const int2 ip = list[e];
-                        const long long src = (((long long)b * p.n_active + ip.x) * p.n_kv_heads + hk) * HD + piece * 8;
-                        dsto[u] = ((long long)bh * p.ctx_len + ip.y) * HD + piece * 8;
-                        v[u] = __ldg(reinterpret_cast<const uint4*>((isv[u] ? p.v_new : p.k_new) + src));
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (isv[u] >= 0) *reinterpret_cast<uint4*>((isv[u] ? p.v_cache : p.k_cache) + dsto[u]) = v[u];
-            }
-            if (chunks > 0) {
-                __threadfence();
-                fence_async_global();   // generic-proxy writes above before this CTA's TMA reads of the same rows
-            }
-            mbar_arrive(bar(B_REFRESHED));
-        }
-
         const int quarter = warp & 3;
         const int kk = quarter * 32 + lane;          // key of the tile == TMEM lane == output column d later on
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const float sl2 = p.scale_log2;
         const f32x2 sl2_2 = pk(sl2, sl2);
-        f32x2 l2[N / 2];
-#pragma unroll
-        for (int i = 0; i < N / 2; ++i) l2[i] = pk(0.f, 0.f);
+        // P^T row of this key: [64-slot half][key][64 slots], 128-byte swizzle
         unsigned char* prow = gbase + p.off_p + (kk >> 3) * 1024 + (kk & 7) * 128;
+        const int bar_or = 2 + 2 * wg, bar_sync = 3 + 2 * wg;   // named barriers of this warpgroup
 
         for (int j = 0; j < T; ++j) {
             mbar_wait(bar(B_SFULL + (j & 1)), (j >> 1) & 1, abort_flag, p.dev_status);
             fence_after();
-            uint32_t sr[N];
-            const uint32_t s_addr = tmem + lane_addr + TM_S + (j & 1) * 64;
-            ld32(s_addr, sr);
-            if (N == 48) ld16(s_addr + 32, sr + 32); else ld32(s_addr + 32, sr + 32);
-            wait_ld();
-            const int key = (t_begin + tile_of(j, spec_ok, rot)) * BK + kk;
-            if (key >= p.ctx_len) {   // only in the ragged last tile of the context
-#pragma unroll
-                for (int c = 0; c < N; ++c) sr[c] = 0xff800000u;   // -inf: probability 0 for every query
-            }
+            const uint32_t s_addr = tmem + lane_addr + TM_S + (j & 1) * NP + c0;
+            const bool past_end = (t_begin + j) * BK + kk >= p.ctx_len;   // only in the ragged last tile of the context
             // d = s * scale * log2(e) - m[q]; does any score exceed its reference by more than 2^8?
-            f32x2 d2[N / 2];
+            f32x2 d2[NH / 2];
+            auto load_d = [&]() {
+                uint32_t sr[NH];
+                ld_row<NH, WG == 1>(s_addr, sr);
+#pragma unroll
+                for (int i = 0; i < NH / 2; ++i) {
+                    const float2 mm = *reinterpret_cast<const float2*>(&sh->m[c0 + 2 * i]);
+                    d2[i] = fma2(pk(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), sl2_2, pk(-mm.x, -mm.y));
+                    if (past_end) d2[i] = pk(-INFINITY, -INFINITY);   // probability 0 for every query
+                }
+            };
+            load_d();
             float dmx0 = -INFINITY, dmx1 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < N / 2; ++i) {
-                const float2 mm = *reinterpret_cast<const float2*>(&sh->m[2 * i]);
-                d2[i] = fma2(pk(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), sl2_2, pk(-mm.x, -mm.y));
+            for (int i = 0; i < NH / 2; ++i) {
                 float d0, d1;
                 upk(d2[i], d0, d1);
                 if (i & 1) dmx1 = max3(dmx1, d0, d1); else dmx0 = max3(dmx0, d0, d1);
             }
-            const bool slow = named_barrier_or(2, kSoft, fmaxf(dmx0, dmx1) > 8.f);
+            const bool slow = named_barrier_or(bar_or, 128, fmaxf(dmx0, dmx1) > 8.f);
+            if (st_w == 0) sh->slow_flag[j & 1][wg] = slow ? 1 : 0;   // for the row-sum threads (read after "P full")
             if (slow) {
-                // ---- rare path: raise the references to the column maxima of this tile, rescale l and O^T ----
+                // ---- rare path: raise the references to the column maxima of this tile, rescale O^T (the row-sum
+                //      threads rescale their sums by the same factors) ----
+                {
+                    uint32_t sr[NH];   // the raw scores once more (they stay in tensor memory until S of tile j + 2)
+                    ld_row<NH, WG == 1>(s_addr, sr);
 #pragma unroll
-                for (int c = 0; c < N; ++c) {
-                    const int o = __reduce_max_sync(0xffffffffu, f2ord(__uint_as_float(sr[c])));
-                    if (lane == (c & 31)) sh->colmax[quarter][c] = o;
+                    for (int c = 0; c < NH; ++c) {
+                        const int o = __reduce_max_sync(0xffffffffu, f2ord(past_end ? -INFINITY : __uint_as_float(sr[c])));
+                        if (lane == (c & 31)) sh->colmax[quarter][c0 + c] = o;
+                    }
                 }
-                named_barrier(3, kSoft);
-                if (stid < N) {
-                    const int o = max(max(sh->colmax[0][stid], sh->colmax[1][stid]), max(sh->colmax[2][stid], sh->colmax[3][stid]));
-                    const float m_old = sh->m[stid];
+                named_barrier(bar_sync, 128);
+                if (st_w < NH) {
+                    const int c = c0 + st_w;
+                    const int o = max(max(sh->colmax[0][c], sh->colmax[1][c]), max(sh->colmax[2][c], sh->colmax[3][c]));
+                    const float m_old = sh->m[c];
                     const float m_new = fmaxf(m_old, ord2f(o) * sl2);
-                    sh->factor[stid] = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - m_new);
-                    sh->m[stid] = m_new;
+                    sh->factor[j & 1][c] = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - m_new);
+                    sh->m[c] = m_new;
                 }
-                named_barrier(3, kSoft);
-#pragma unroll
-                for (int i = 0; i < N / 2; ++i) {
-                    const float2 ff = *reinterpret_cast<const float2*>(&sh->factor[2 * i]);
-                    l2[i] = mul2(l2[i], pk(ff.x, ff.y));
-                }
+                named_barrier(bar_sync, 128);
                 if (j > 0) {   // O^T holds the tiles before j: P V of tile j - 1 must have completed
                     mbar_wait(bar(B_PVDONE), (j - 1) & 1, abort_flag, p.dev_status);
                     fence_after();
-                    uint32_t o[N];
-                    const uint32_t o_addr = tmem + lane_addr + TM_O;
-                    ld32(o_addr, o);
-                    if (N == 48) ld16(o_addr + 32, o + 32); else ld32(o_addr + 32, o + 32);
-                    wait_ld();
+                    uint32_t o[NH];
+                    const uint32_t o_addr = tmem + lane_addr + TM_O + c0;
+                    ld_row<NH, WG == 1>(o_addr, o);
 #pragma unroll
-                    for (int c = 0; c < N; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * sh->factor[c]);
-                    st32(o_addr, o);
-                    if (N == 48) st16(o_addr + 32, o + 32); else st32(o_addr + 32, o + 32);
-                    wait_st();
+                    for (int c = 0; c < NH; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * sh->factor[j & 1][c0 + c]);
+                    st_row<NH, WG == 1>(o_addr, o);
                 }
-#pragma unroll
-                for (int i = 0; i < N / 2; ++i) {
-                    const float2 mm = *reinterpret_cast<const float2*>(&sh->m[2 * i]);
-                    d2[i] = fma2(pk(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), sl2_2, pk(-mm.x, -mm.y));
-                }
+                load_d();   // against the raised references
             }
-            uint32_t pw[N / 2];
+            uint32_t pw[NH / 2];
 #pragma unroll
-            for (int i = 0; i < N / 2; ++i) {
+            for (int i = 0; i < NH / 2; ++i) {
                 float d0, d1;
                 upk(d2[i], d0, d1);
-                const float e0 = fast_exp2(d0), e1 = fast_exp2(d1);
-                l2[i] = add2(l2[i], pk(e0, e1));
-                pw[i] = pack_bf16x2(e0, e1);
+                pw[i] = pack_bf16x2(fast_exp2(d0), fast_exp2(d1));
             }
-            // the P^T buffer is free once P V of the previous tile has completed
-            if (j > 0) mbar_wait(bar(B_PVDONE), (j - 1) & 1, abort_flag, p.dev_status);
+            // the P^T buffer is free once P V of the previous tile has completed and its row sums have been taken
+            if (j > 0) {
+                mbar_wait(bar(B_PVDONE), (j - 1) & 1, abort_flag, p.dev_status);
+                mbar_wait(bar(B_PSUM), (j - 1) & 1, abort_flag, p.dev_status);
+            }
 #pragma unroll
-            for (int ch = 0; ch < N / 8; ++ch)
-                *reinterpret_cast<uint4*>(prow + ((ch ^ (kk & 7)) << 4)) = make_uint4(pw[4 * ch], pw[4 * ch + 1], pw[4 * ch + 2], pw[4 * ch + 3]);
+            for (int ch = 0; ch < NH / 8; ++ch) {
+                const int gch = (c0 >> 3) + ch;      // 16-byte chunk (8 slots) of the whole P^T row
+                *reinterpret_cast<uint4*>(prow + (gch >> 3) * SUB + (((gch & 7) ^ (kk & 7)) << 4)) =
+                    make_uint4(pw[4 * ch], pw[4 * ch + 1], pw[4 * ch + 2], pw[4 * ch + 3]);
+            }
             fence_async_smem();
             fence_before();
             mbar_arrive(bar(B_PFULL));
@@ -502,115 +522,111 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         mbar_wait(bar(B_PVDONE), (T - 1) & 1, abort_flag, p.dev_status);   // Q, P^T and the K/V stages are dead from here on
         fence_after();
         if (C > 1) {
-            // first cluster barrier, arrive half: from here on the peers may write their partials into this CTA's
-            // receive buffer (dead stage memory that the reduction and the staging below do not touch)
+            // first cluster barrier, arrive half: the peers may write their partials into this CTA's receive chunks
             __syncwarp();
             cluster_arrive();
         }
+        mbar_wait(bar(B_PSUM), (T - 1) & 1, abort_flag, p.dev_status);     // the row sums are complete
 
-        // ---- row sums over the CTA's keys: per-thread partials -> shared memory -> one thread per query ----
-        float* lred = reinterpret_cast<float*>(gbase);   // [128 keys][NP]
-#pragma unroll
-        for (int i = 0; i < N / 2; ++i) {
-            float a0, a1;
-            upk(l2[i], a0, a1);
-            lred[kk * NP + 2 * i] = a0;
-            lred[kk * NP + 2 * i + 1] = a1;
-        }
-        named_barrier(3, kSoft);
-        {   // two threads per query column, 64 keys each
-            const int qc = stid & 63, half = stid >> 6;
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            if (qc < N) {
-#pragma unroll
-                for (int k = 0; k < 64; ++k) acc[k & 7] += lred[(half * 64 + k) * NP + qc];
-            }
-            const float part = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
-            named_barrier(3, kSoft);   // every partial sum has been read out of lred
-            if (qc < N) lred[half * N + qc] = part;
-            named_barrier(3, kSoft);
-            if (stid < N) sh->factor[stid] = lred[stid] + lred[N + stid];   // l[q] of this CTA
-        }
-        named_barrier(3, kSoft);
-
-        uint32_t o[N];
-        {
-            const uint32_t o_addr = tmem + lane_addr + TM_O;
-            ld32(o_addr, o);
-            if (N == 48) ld16(o_addr + 32, o + 32); else ld32(o_addr + 32, o + 32);
-            wait_ld();
-        }
+        uint32_t o[NH];
+        ld_row<NH, WG == 1>(tmem + lane_addr + TM_O + c0, o);
         if (C == 1) {
             // ---- single CTA per (sequence, kv head): normalise and store column kk of every query row ----
+            if (!*abort_flag) {
 #pragma unroll
-            for (int c = 0; c < N; ++c) {
-                if (c < rows_total) {
-                    const int i = i0 + c / p.group, jh = c % p.group;
-                    __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD;
-                    dst[kk] = __float2bfloat16_rn(__uint_as_float(o[c]) / sh->factor[c]);
+                for (int c = 0; c < NH; ++c) {
+                    if (c0 + c < rows_total) {
+                        const float l = sh->lpart[0][c0 + c] + (kParts == 2 ? sh->lpart[1][c0 + c] : 0.f);
+                        const int i = i0 + (c0 + c) / p.group, jh = (c0 + c) % p.group;
+                        __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD;
+                        dst[kk] = __float2bfloat16_rn(__uint_as_float(o[c]) / l);
+                    }
                 }
             }
         } else {
-            // ---- this CTA's O^T row kk -> staging chunk of the CTA that owns output column kk ----
-            float* stg = reinterpret_cast<float*>(gbase + kStagingOff) + (kk / DL) * (chunk_bytes / 4) + (kk % DL) * NP;
+            // ---- this thread's O^T row (output column kk, its warpgroup's queries) -> the staging chunk of the
+            //      CTA that owns column kk; consecutive lanes write consecutive words ----
+            float* stg = reinterpret_cast<float*>(gbase + stg_off) + (kk / DL) * chunk_floats + (kk % DL);
 #pragma unroll
-            for (int c = 0; c < N; ++c) stg[c] = __uint_as_float(o[c]);
-            if (stid < N) {   // every owner also gets this CTA's m[q] and l[q]
-                for (int c = 0; c < C; ++c) {
-                    float* ml = reinterpret_cast<float*>(gbase + kStagingOff) + c * (chunk_bytes / 4) + DL * NP;
-                    ml[stid] = sh->m[stid];
-                    ml[N + stid] = sh->factor[stid];
+            for (int c = 0; c < NH; ++c)
+                if (c0 + c < rows_total) stg[(c0 + c) * DL] = __uint_as_float(o[c]);
+            if (st_w < NH) {   // every owner also gets this CTA's m[q] and l[q]
+                const int c = c0 + st_w;
+                const float l = sh->lpart[0][c] + (kParts == 2 ? sh->lpart[1][c] : 0.f);
+                for (int ow = 0; ow < C; ++ow) {
+                    float* ml = reinterpret_cast<float*>(gbase + stg_off) + ow * chunk_floats + N * DL;
+                    ml[c] = sh->m[c];
+                    ml[N + c] = l;
                 }
             }
             fence_async_smem();   // staging (generic proxy) -> bulk copies (async proxy)
+            named_barrier(6, kSoft);
+            __syncwarp();
+            cluster_wait();       // every CTA of the cluster is past its main loop
+            if (stid < C) {       // one bulk copy per owner into the owner's receive chunk of this source
+                const uint32_t src = base + stg_off + (uint32_t)stid * chunk_bytes;
+                const uint32_t dst = map_to_cta(base + recv_off + (uint32_t)split * chunk_bytes, stid);
+                bulk_copy_to_peer(dst, src, chunk_bytes, map_to_cta(bar(B_RECV), stid));
+            }
         }
-        fence_before();
     }
 
     if (C > 1) {
-        // the slices are staged (CTA barrier: the softmax warps wrote them, warp 0 sends them) and every CTA of
-        // the cluster is past its main loop (its Q, P^T and K/V stages are dead, its barriers initialised)
-        __syncthreads();
-        cluster_wait();
-        if (warp == 0 && lane < C) {   // one bulk copy per owner into the owner's receive buffer
-            const uint32_t src = base + kStagingOff + (uint32_t)lane * chunk_bytes;
-            const uint32_t dst = map_to_cta(base + kRecvOff + (uint32_t)split * chunk_bytes, lane);
-            bulk_copy_to_peer(dst, src, chunk_bytes, map_to_cta(bar(B_RECV), lane));
+        if (!(warp >= 2 && warp < 2 + 4 * WG)) {   // the other warps' halves of the first cluster barrier
+            __syncwarp();
+            cluster_arrive();
+            cluster_wait();
         }
         // ---- merge the C partials of the output columns this CTA owns -------------------------
         mbar_wait(bar(B_RECV), 0, abort_flag, p.dev_status);
-        // second cluster barrier, arrive half: this CTA holds every peer's partial, i.e. the peers' copies out of
-        // their staging areas have completed; the wait half, before leaving, overlaps the merge
+        // second cluster barrier, arrive half: this CTA holds every peer's partial, so the peers' copies out of their
+        // staging chunks have completed; the wait half, before leaving, overlaps the merge
         __syncwarp();
         cluster_arrive();
-        const float* recv = reinterpret_cast<const float*>(gbase + kRecvOff);
-        const int cf = (int)(chunk_bytes / 4);
-        float* wgt = reinterpret_cast<float*>(gbase);   // [C][N] normalised weights 2^(m_s - m) / l, over the dead row-sum scratch
-        long long* qoff = reinterpret_cast<long long*>(gbase + 4096);   // [N] element offset of each query row in out
-        if (tid < N) {
-            float m = -INFINITY;
-            for (int s = 0; s < C; ++s) m = fmaxf(m, recv[s * cf + DL * NP + tid]);
-            float l = 0.f;
-            for (int s = 0; s < C; ++s) l = fmaf(fast_exp2(recv[s * cf + DL * NP + tid] - m), recv[s * cf + DL * NP + N + tid], l);
-            const float inv = 1.f / l;
-            for (int s = 0; s < C; ++s) wgt[s * N + tid] = fast_exp2(recv[s * cf + DL * NP + tid] - m) * inv;
+        const float* recv = reinterpret_cast<const float*>(gbase + recv_off);
+        float* wgt = reinterpret_cast<float*>(gbase + wgt_off);                  // [8][N] weights 2^(m_s - m) / l
+        long long* qoff = reinterpret_cast<long long*>(gbase + qoff_off);        // [N] element offset of each query row in out
+        // weights: eight lanes per query row, one per source
+        for (int it0 = 0; it0 < rows_total * 8; it0 += kThreads) {
+            const int it = it0 + tid, q = it >> 3, s = it & 7;
+            const bool live = q < rows_total && s < C;
+            const float ms = live ? recv[s * chunk_floats + N * DL + q] : -INFINITY;
+            const float ls = live ? recv[s * chunk_floats + N * DL + N + q] : 0.f;
+            float m = ms;
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+            const float e = live ? fast_exp2(ms - m) : 0.f;
+            float l = e * ls;
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            l += __shfl_xor_sync(0xffffffffu, l, 4);
+            if (live) wgt[s * N + q] = e / l;
+        }
+        if (tid < rows_total) {
             const int i = i0 + tid / p.group, jh = tid % p.group;
             qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL;
         }
         __syncthreads();
         // a thread owns two adjacent output columns of a query row: one 4-byte store
-        const int half_dl = DL / 2;
-        const int dp = tid % half_dl;
-        for (int qq = tid / half_dl; qq < rows_total; qq += kThreads / half_dl) {
-            float a0 = 0.f, a1 = 0.f;
-            for (int s = 0; s < C; ++s) {
-                const float w = wgt[s * N + qq];
-                a0 = fmaf(w, recv[s * cf + (2 * dp) * NP + qq], a0);
-                a1 = fmaf(w, recv[s * cf + (2 * dp + 1) * NP + qq], a1);
+        const int half_dl = min(DL, HD - split * DL) / 2;
+        if (!*abort_flag) {
+            for (int idx = tid; idx < rows_total * half_dl; idx += kThreads) {
+                const int qq = idx / half_dl, dp = idx % half_dl;
+                float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    if (s < C) {
+                        const float w = wgt[s * N + qq];
+                        const float2 v = *reinterpret_cast<const float2*>(recv + s * chunk_floats + qq * DL + 2 * dp);
+                        a0 = fmaf(w, v.x, a0);
+                        a1 = fmaf(w, v.y, a1);
+                    }
+                }
+                *reinterpret_cast<uint32_t*>(p.out + qoff[qq] + 2 * dp) = pack_bf16x2(a0, a1);
             }
-            *reinterpret_cast<uint32_t*>(p.out + qoff[qq] + 2 * dp) = pack_bf16x2(a0, a1);
         }
-        // no CTA leaves while a peer may still copy out of or into its shared memory
+        // no CTA leaves while a peer may still copy out of its staging chunks
         __syncwarp();
         cluster_wait();
     }
@@ -624,23 +640,6 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
 }
 
 // ---- host side ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
 // cache [B*Hkv, L, 128] bf16 seen as 4-D {64 columns, key, half, head}: one box {64, 128, 2, 1} lands as
 // [half][key][64 columns], the two 128-byte-swizzled halves of a [128 keys x 128] tile; keys beyond L read as zero
 bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
@@ -655,7 +654,7 @@ bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// q [B, n, H_q, 128] bf16 (MHA: one query head per kv head) seen as 5-D {64 columns, row, head, half, sequence}:
+// q [B, n, H_q, 128] bf16 (one query head per CTA column) seen as 5-D {64 columns, row, head, half, sequence}:
 // the box {64, N, 1, 2, 1} lands as [half][row][64 columns], the K-major Q tile; rows past n read as zero
 bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_q_heads, int n_slots) {
     EncodeTiledFn fn = encode_fn();
@@ -671,55 +670,88 @@ bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_
 }
 
 struct KeysPlan {
+    bool ok;
     int group, rows_chunk, n_sub_r, n_sub;   // heads and active rows per CTA column, row chunks, CTA columns per kv head
-    int n_slots, n_splits, tiles_per_split, n_stages;
+    int n_slots, n_splits, tiles_per_split, n_stages, dl, ctas_per_sm;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
 };
 
-constexpr uint32_t kSmemMax = 232448;   // 227 KB: largest dynamic allocation of one CTA
+constexpr uint32_t kSmemMax = 232448;        // 227 KB: largest dynamic allocation of one CTA
+constexpr uint32_t kSmemTwoPerSm = 115712;   // (228 KB per SM - 2 x 1 KB reserved) / 2
+
+// tensor-memory columns the instantiation for n_slots allocates (see TM_COLS in the kernel)
+constexpr int tm_columns(int n_slots) { return 3 * (n_slots <= 64 ? 64 : 128) <= 256 ? 256 : 512; }
+
+// shared-memory carve for n_slots query slots and ns stages
+void carve(KeysPlan& pl, int n_active, int ns) {
+    uint32_t off = (uint32_t)pl.n_slots * 256u;   // Q
+    off = (off + 1023u) & ~1023u;
+    pl.off_p = off;
+    off += (uint32_t)((pl.n_slots + 63) / 64) * SUB;
+    pl.off_stage = off;
+    off += (uint32_t)ns * STAGE;
+    pl.off_list = off;
+    off += ((uint32_t)n_active * 8u + 15u) & ~15u;
+    pl.off_bar = off;
+    off += kBarBytes + (uint32_t)sizeof(KeysShared) + 16u;
+    pl.smem_bytes = off + 1024u;
+    // an instantiation that allocates all 512 columns of tensor memory must never share an SM with a CTA of its own
+    // cluster (the second allocation would wait for the first CTA, which waits for it at the cluster barrier): ask for
+    // more than half an SM's shared memory
+    if (tm_columns(pl.n_slots) > 256 && pl.smem_bytes <= kSmemTwoPerSm) pl.smem_bytes = kSmemTwoPerSm + 1024u;
+    pl.n_stages = ns;
+}
 
 KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
     KeysPlan pl{};
-    // a CTA column takes the largest divisor of the H_q / H_kv heads of a kv head whose packed rows fit the 64
-    // query slots; the other columns of that kv head stream the same K/V (from L2) for their own heads
+    // a CTA column takes the largest divisor of the H_q / H_kv heads of a kv head whose packed rows fit the query
+    // slots; the other columns of that kv head stream the same K/V (from L2) for their own heads
     const int g = d.n_q_heads / d.n_kv_heads;
     pl.group = g;
-    while (pl.group > 1 && (g % pl.group != 0 || (long long)n_active * pl.group > kMaxRowsT)) --pl.group;
-    // more active rows than slots (the paper's default budget k = 64 gives 96): the rows are cut into equal chunks,
-    // one CTA column each
-    pl.n_sub_r = (n_active * pl.group + kMaxRowsT - 1) / kMaxRowsT;
+    while (pl.group > 1 && (g % pl.group != 0 || (long long)n_active * pl.group > kMaxSlots)) --pl.group;
+    // more active rows than slots: the rows are cut into equal chunks, one CTA column each
+    pl.n_sub_r = (n_active * pl.group + kMaxSlots - 1) / kMaxSlots;
     pl.rows_chunk = (n_active + pl.n_sub_r - 1) / pl.n_sub_r;
     pl.n_sub_r = (n_active + pl.rows_chunk - 1) / pl.rows_chunk;
     pl.n_sub = (g / pl.group) * pl.n_sub_r;
     const int rows = pl.rows_chunk * pl.group;
-    pl.n_slots = rows <= 48 ? 48 : 64;
+    pl.n_slots = rows <= 48 ? 48 : rows <= 64 ? 64 : 96;
+    const int tm_cols = tm_columns(pl.n_slots);
     const int key_tiles = (d.ctx_len + BK - 1) / BK;
-    const int bh = d.batch * d.n_kv_heads * pl.n_sub;
-    // one CTA per SM; the cluster size divides the 128 output columns, every CTA gets at least one tile
-    int c = 1;
-    while (c < 8 && 2 * c * bh <= sm_count() && 2 * c <= key_tiles) c *= 2;
-    pl.tiles_per_split = (key_tiles + c - 1) / c;
-    while (c > 1 && (key_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split < c) {   // no empty CTA
-        c /= 2;
-        pl.tiles_per_split = (key_tiles + c - 1) / c;
+    const long long columns = (long long)d.batch * d.n_kv_heads * pl.n_sub;   // grid.y
+    const int sms = sm_count();
+    // cluster size: every CTA at least one tile, all CTAs resident at once (two per SM when they are small), and
+    // the most-loaded SM streaming as few tiles as possible; among equals, more CTAs (more SMs pulling)
+    long long best_load = -1, best_ctas = 0;
+    for (int c = 1; c <= 8 && c <= key_tiles; ++c) {
+        const int tps = (key_tiles + c - 1) / c;
+        if ((key_tiles + tps - 1) / tps != c || tps > kMaxTiles) continue;   // this c leaves a CTA empty
+        int dl = (HD + c - 1) / c;
+        dl += dl & 1;
+        if ((c - 1) * dl >= HD) continue;                                    // an owner without columns
+        KeysPlan t = pl;
+        int ns = tps < kMaxStages ? tps : kMaxStages;
+        carve(t, n_active, ns);
+        while (ns > 1 && t.smem_bytes > kSmemMax) carve(t, n_active, --ns);
+        if (t.smem_bytes > kSmemMax || (ns < 2 && tps > 1)) continue;
+        // the exchange areas of the merge (2 c chunks, weights, row offsets) reuse the Q / P^T / stage memory
+        if (c > 1 && 2 * (size_t)c * (pl.n_slots * dl + 2 * pl.n_slots) * 4 + (size_t)pl.n_slots * 40 > t.off_list) continue;
+        const int per_sm = (t.smem_bytes <= kSmemTwoPerSm && tm_cols <= 256) ? 2 : 1;
+        const long long ctas = columns * c;
+        if (ctas > (long long)per_sm * sms) continue;
+        const long long load = (long long)tps * ((ctas + sms - 1) / sms);
+        if (best_load < 0 || load < best_load || (load == best_load && ctas > best_ctas)) {
+            best_load = load;
+            best_ctas = ctas;
+            pl.n_splits = c;
+            pl.tiles_per_split = tps;
+            pl.dl = dl;
+            pl.ctas_per_sm = per_sm;
+            pl.n_stages = ns;
+        }
     }
-    pl.n_splits = c;
-    uint32_t off = (uint32_t)pl.n_slots * 256u;   // Q
-    pl.off_p = off;
-    off += P_BYTES;
-    pl.off_stage = off;
-    const uint32_t list = ((uint32_t)n_active * 8u + 15u) & ~15u;
-    const uint32_t tail = list + B_COUNT * 8u + (uint32_t)sizeof(KeysShared) + 16u + 1024u;
-    int ns = (int)((kSmemMax - off - tail) / STAGE);
-    if (ns > kMaxStages) ns = kMaxStages;
-    if (ns > pl.tiles_per_split && ns > 2) ns = pl.tiles_per_split < 2 ? 2 : pl.tiles_per_split;
-    pl.n_stages = ns;
-    off += (uint32_t)ns * STAGE;
-    pl.off_list = off;
-    off += list;
-    pl.off_bar = off;
-    off += B_COUNT * 8u + (uint32_t)sizeof(KeysShared) + 16u;
-    pl.smem_bytes = off + 1024u;
+    pl.ok = best_load >= 0;
+    if (pl.ok) carve(pl, n_active, pl.n_stages);
     return pl;
 }
 
@@ -731,7 +763,7 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
         return ea;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(pl.n_splits, bh, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + kAuxThreads, 1, 1);
     cfg.dynamicSmemBytes = pl.smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];
@@ -752,24 +784,23 @@ bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
     if (n_active > kMaxActive) return false;
     const KeysPlan pl = make_keys_plan(d, n_active);
+    if (!pl.ok) return false;   // no cluster size keeps all CTAs resident: the row-major skip kernel streams better
     if ((long long)d.batch * d.n_kv_heads * pl.n_sub > 65535) return false;   // grid.y
-    // the exchange areas (row-sum scratch, staging, receive buffer) reuse the memory below the refresh list
-    // one CTA per SM: beyond one wave of CTAs the row-major skip kernel (two CTAs per SM) streams better
-    if ((long long)pl.n_splits * d.batch * d.n_kv_heads * pl.n_sub > sm_count()) return false;
     // row chunks re-read the K/V of a head once per chunk: only worth it while the keys can still be split
     if (pl.n_sub_r > 1 && pl.n_splits < 2) return false;
-    return pl.n_stages >= 2 && pl.smem_bytes <= kSmemMax && kRecvOff + kExchangeMax <= pl.off_list;
+    return true;
 }
 
 void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
     const KeysPlan pl = make_keys_plan(d, n_active);
-    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u", pl.n_slots, pl.n_splits,
-             d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes);
+    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u ctas_per_sm=%d", pl.n_slots,
+             pl.n_splits, d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes, pl.ctas_per_sm);
 }
 
 cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                     cudaStream_t stream) {
     const KeysPlan pl = make_keys_plan(a.d, a.n_active);
+    if (!pl.ok) return cudaErrorInvalidConfiguration;
     const int bh = a.d.batch * a.d.n_kv_heads;
     CUtensorMap map_k, map_v;
     if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
@@ -797,13 +828,16 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.n_splits = pl.n_splits;
     p.tiles_per_split = pl.tiles_per_split;
     p.n_stages = pl.n_stages;
+    p.dl = pl.dl;
     p.off_p = pl.off_p;
     p.off_stage = pl.off_stage;
     p.off_list = pl.off_list;
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
-    return pl.n_slots == 48 ? launch_n<48>(pl, p, map_k, map_v, map_q, bh * pl.n_sub, stream)
-                            : launch_n<64>(pl, p, map_k, map_v, map_q, bh * pl.n_sub, stream);
+    const int cols = bh * pl.n_sub;
+    return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, cols, stream)
+           : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, cols, stream)
+                              : launch_n<96>(pl, p, map_k, map_v, map_q, cols, stream);
 }
 
 }  // namespace ec

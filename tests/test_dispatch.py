@@ -18,9 +18,9 @@ SKIP_STEP = [
     ("c5_llada_l4096", 5, 34, "attend_skip_kernel<1>"),
     ("c4_dream_l2048", None, 34, "attend_skip_keys_kernel<48>"),
     ("c5_dream_l4096", None, 34, "attend_skip_keys_kernel<48>"),
-    ("c5_llada_l4096", None, 96, "attend_skip_keys_kernel<48>"),    # the paper's default budget k = 64
+    ("c5_llada_l4096", None, 96, "attend_skip_keys_kernel<96>"),    # the paper's default budget k = 64
     ("c5_llada_l4096_b8", None, 96, "attend_skip_kernel<1>"),
-    ("c5_dream_l4096", None, 96, "attend_skip_keys_kernel<48>"),
+    ("c5_dream_l4096", None, 96, "attend_skip_keys_kernel<96>"),
     ("c1_tiny_fp32", None, 34, "refresh_kernel + attend_f32_kernel"),
 ]
 
@@ -70,10 +70,15 @@ def test_other_instantiations_and_fallbacks_are_reachable():
 
     assert name(2, 1000, 8, 8, 128, syn.BF16, 56).startswith("attend_skip_keys_kernel<64>")
     assert name(2, 333, 6, 3, 128, syn.BF16, 100).startswith("attend_skip_keys_kernel<64>")  # 200 packed rows
-    assert name(1, 640, 4, 4, 128, syn.BF16, 256).startswith("attend_skip_keys_kernel<64>")  # four row chunks
-    assert name(1, 2048, 32, 32, 128, syn.BF16, 160).startswith("attend_skip_kernel<2> grid=(4,32) cluster=4")
+    assert name(1, 640, 4, 4, 128, syn.BF16, 256).startswith("attend_skip_keys_kernel<96>")  # three row chunks
+    assert name(1, 768, 32, 32, 128, syn.BF16, 34).startswith("attend_skip_keys_kernel<48> grid=(6,32) cluster=6")
+    assert "ctas_per_sm=2" in name(1, 768, 32, 32, 128, syn.BF16, 34)                     # one tile per CTA, two CTAs per SM
+    assert name(1, 4096, 28, 4, 128, syn.BF16, 34).startswith("attend_skip_keys_kernel<48> grid=(5,28) cluster=5")
+    assert name(2, 768, 32, 32, 128, syn.BF16, 128).startswith("attend_skip_kernel<1> grid=(4,64) cluster=4")
+    assert name(3, 768, 32, 32, 128, syn.BF16, 128).startswith("attend_skip_kernel<1> grid=(3,96) cluster=3")
+    assert name(2, 768, 32, 32, 128, syn.BF16, 160).startswith("attend_skip_kernel<2> grid=(2,64) cluster=2")
     assert name(8, 4096, 32, 32, 128, syn.BF16, 200).startswith("attend_skip_kernel<2> grid=(1,256) cluster=1")
-    assert name(2, 65, 6, 3, 128, syn.BF16, 65, idx=False) == "refresh_kernel + attend_tc_kernel"
+    assert name(2, 65, 6, 3, 128, syn.BF16, 65, idx=False).startswith("attend_skip_keys_kernel<96> grid=(1,12) cluster=1")
     assert name(2, 259, 4, 2, 128, syn.BF16, 259, idx=False) == "refresh_kernel + attend_tc_kernel"
     assert name(2, 130, 6, 3, 64, syn.BF16, 17) == "refresh_kernel + attend_mma_kernel"
     assert name(2, 130, 6, 3, 64, syn.F32, 17) == "refresh_kernel + attend_f32_kernel"

@@ -166,14 +166,33 @@ def test_grouped_query_skip_steps_spread_over_head_columns(Hq, Hkv, n, L):
 @pytest.mark.parametrize("Hq,Hkv,n,L", [(32, 32, 96, 768), (8, 8, 70, 1000), (4, 4, 256, 640), (28, 4, 96, 768),
                                         (6, 2, 129, 515), (16, 16, 160, 2048)])
 def test_skip_steps_with_more_active_rows_than_query_slots(Hq, Hkv, n, L):
-    """The paper's default budget k = 64 gives 96 active rows, its grid up to 288: the active rows are cut into
-    chunks of at most 64 packed rows, one CTA column each (48 + 48 at n = 96, 35 + 35 at n = 70, four chunks at
-    256, with GQA on top: 2 row chunks x 7 head columns), every column refreshing the whole list's rows."""
+    """The paper's default budget k = 64 gives 96 active rows, its grid up to 288: up to 96 packed rows share one
+    CTA column (two softmax warpgroups split the columns of a key), beyond that the active rows are cut into equal
+    chunks, one CTA column each (80 + 80 at n = 160, three chunks at 256, with GQA on top: 7 head columns), every
+    column patching the whole list's rows into its tiles."""
     w = syn.Workload(96, "row_chunks", syn.BF16, 1, Hq, Hkv, 128, 0, L, 1, 0, 64)
     idx = syn.arbitrary_active_idx(1, L, n, seed=13 * L + n)
     t = syn.attn_inputs(w, n, active_idx=idx, std_qk=0.7, std_v=0.5)
     _check(w, t)
     _check(w, t, refresh=False)
+
+
+@pytest.mark.parametrize("B,n,kernel", [(2, 128, "attend_skip_kernel<1> grid=(4,64) cluster=4"),
+                                        (3, 128, "attend_skip_kernel<1> grid=(3,96) cluster=3"),
+                                        (2, 160, "attend_skip_kernel<2> grid=(2,64) cluster=2"),
+                                        (2, 192, "attend_skip_kernel<2> grid=(2,64) cluster=2")])
+def test_many_row_skip_steps_on_the_row_major_kernel_with_clusters(B, n, kernel):
+    """Skip steps of several sequences with 128 to 192 active rows (the upper half of the paper's budget grid): the
+    kernel with the query rows on the M axis, one and two row tiles, the keys of a head split over a cluster of two
+    to four CTAs that exchange their partial rows."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.Workload(92, "rows_clusters", syn.BF16, B, 32, 32, 128, 0, 768, 1, 0, 64)
+    d = ec.make_desc(B, 768, 32, 32, 128, syn.BF16)
+    assert ec.ec_attend_kernel_name(d, n, True, True).startswith(kernel)
+    idx = syn.arbitrary_active_idx(B, 768, n, seed=17 * n + B)
+    t = syn.attn_inputs(w, n, active_idx=idx, std_qk=0.7, std_v=0.5)
+    _check(w, t)
 
 
 def test_few_row_skip_step_with_rising_maxima():
