@@ -47,7 +47,9 @@ int forced_impl() {
     return f;
 }
 bool use_tc(const ec_attn_desc& d) { return d.dtype == EC_BF16 && d.head_dim == 128 && forced_impl() != 1; }
-bool use_skip_keys(const ec_attn_desc& d, int n_active) { return forced_impl() == 0 && attend_skip_keys_supported(d, n_active); }
+bool use_skip_keys(const ec_attn_desc& d, int n_active, bool fresh) {
+    return forced_impl() == 0 && attend_skip_keys_supported(d, n_active, fresh);
+}
 bool use_skip(const ec_attn_desc& d, int n_active) {
     return (forced_impl() == 0 || forced_impl() == 3) && attend_skip_supported(d, n_active);
 }
@@ -66,7 +68,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // which kernel serves a call of ec_attend: the one place the dispatch order is written down
 enum AttendPath { PATH_SKIP_KEYS, PATH_SKIP_ROWS, PATH_DENSE_FROM_NEW, PATH_DENSE, PATH_TC_ONE_TILE, PATH_MMA, PATH_F32 };
 AttendPath choose_path(const ec_attn_desc& d, int n_active, bool fresh_kv, bool index_list) {
-    if (use_skip_keys(d, n_active)) return PATH_SKIP_KEYS;
+    if (use_skip_keys(d, n_active, fresh_kv)) return PATH_SKIP_KEYS;
     if (use_skip(d, n_active)) return PATH_SKIP_ROWS;
     if (d.dtype != EC_BF16) return PATH_F32;
     if (use_tc(d) && forced_impl() != 2 && attend_dense_supported(d, n_active))
@@ -245,7 +247,7 @@ const char* ec_attend_kernel_name(const ec_attn_desc* desc, int32_t n_active, in
         return "";
     const bool fresh = with_fresh_kv != 0;
     switch (choose_path(*desc, n_active, fresh, with_index_list != 0)) {
-        case PATH_SKIP_KEYS: attend_skip_keys_describe(*desc, n_active, buf, sizeof buf); return buf;
+        case PATH_SKIP_KEYS: attend_skip_keys_describe(*desc, n_active, fresh, buf, sizeof buf); return buf;
         case PATH_SKIP_ROWS: attend_skip_describe(*desc, n_active, buf, sizeof buf); return buf;
         case PATH_F32: return fresh ? "refresh_kernel + attend_f32_kernel" : "attend_f32_kernel";
         case PATH_DENSE_FROM_NEW: attend_dense_describe(*desc, n_active, buf, sizeof buf); return buf;

@@ -25,24 +25,28 @@
 //            the rows) are spread over n_sub CTA columns that stream the same K/V (L2 serves the repeats);
 //   K/V      the producer warp issues its TMA loads at once, in key order, through a ring of NS stages of 64 KB:
 //            they depend on nothing;
-//   refresh  the active rows' fresh K/V reach the attention through SHARED memory, not through the cache: two
-//            patch warps copy the fresh rows of the CTA's key range from k_new / v_new over the stale rows of the
-//            landed tile (same swizzled layout the TMA wrote) before that tile's first product is issued, and
-//            write the same bytes into the cache in global memory for later steps.  Whether a concurrent TMA
-//            read of such a row saw the old or the new bytes does not matter, so nothing orders the cache update
-//            against the loads;
+//   refresh  the active rows' fresh K/V reach the attention straight from k_new / v_new, not through the cache: one
+//            CTA of every cluster (the last) attends to them as one or two EXTRA key tiles, fetched by TMA from the
+//            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) before its cache
+//            tiles, while every CTA masks the stale cached keys of the refreshed positions (a bit per key, built from
+//            the index list).  The attention therefore never waits for the cache update: the auxiliary warps of that
+//            CTA copy the fresh rows into the cache in global memory for later steps, ordered against nothing.  (Keys
+//            in a different order, the same sum.)  When a CTA holds a single cache tile the extra tiles get a CTA of
+//            their own, so that nobody streams two tiles through one stage;
 //   merge    CTA c of the cluster owns the output columns d in [c*DL, (c+1)*DL): once every CTA of the cluster is
 //            past its main loop (first cluster barrier) each softmax thread stores its O^T row (one output column,
 //            all queries) straight into the owner's shared memory, plus m and l; after the second cluster barrier
 //            the owner combines the C partials, normalises and writes out[b, i, h, d].
-// warp 0: TMA producer; warp 1: refresh list, then tcgen05.mma issue; next 4 (or 8) warps: softmax; last two
-// warps: patch / refresh.  Launched with programmatic stream serialisation; global memory is touched only after
+// warp 0: TMA producer; warp 1: stale-key masks, then tcgen05.mma issue; next 4 (or 8) warps: softmax; last two
+// warps: cache update and row sums.  Launched with programmatic stream serialisation; global memory is touched only after
 // griddepcontrol.wait.  Every mbarrier wait is bounded (EC_ERR_TIMEOUT in dev_status, CTA-wide abort flag: an
 // aborted CTA stores no output); the CTA always frees its TMEM and exits.
 #include "ec_common.cuh"
 #include "ec_tc_ptx.cuh"
 
 #include <cstdio>
+#include <mutex>
+#include <vector>
 
 namespace ec {
 namespace {
@@ -50,8 +54,7 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 128, HD = 128;
-constexpr int kAuxThreads = 64;           // two warps: refresh patches and row sums
-constexpr int kPatchPer = 18;             // 16-byte pieces of fresh rows a thread holds per round (36 rows per round)
+constexpr int kAuxThreads = 64;           // two warps: cache update and row sums
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr uint32_t STAGE = 2 * TILE;       // K tile + V tile: 64 KB
@@ -61,8 +64,8 @@ constexpr int kMaxActive = 256;            // active rows of a sequence (refresh
 constexpr int kMaxTiles = 1024;            // key tiles of one CTA (bits of the patch mask)
 
 enum { B_FULL = 0, B_EMPTY = kMaxStages, B_SFULL = 2 * kMaxStages, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 1,
-       B_PSUM = B_PVDONE + 1, B_QFULL = B_PSUM + 1, B_LIST = B_QFULL + 1, B_NEEDPATCH = B_LIST + 1,
-       B_PATCHED = B_NEEDPATCH + kMaxStages, B_RECV = B_PATCHED + kMaxStages, B_COUNT = B_RECV + 1 };
+       B_PSUM = B_PVDONE + 1, B_QFULL = B_PSUM + 1, B_LIST = B_QFULL + 1, B_FRESHOUT = B_LIST + 1, B_RECV = B_FRESHOUT + 2,
+       B_COUNT = B_RECV + 1 };
 
 constexpr uint32_t kBarBytes = (B_COUNT * 8u + 15u) & ~15u;   // the barrier block, padded so that what follows is 16-byte aligned
 
@@ -114,9 +117,11 @@ struct KeysParams {
     int n_sub_r;      // row chunks = ceil(n_active / rows_chunk)
     int n_sub;        // CTA columns per kv head = ((H_q / H_kv) / group) * n_sub_r
     int n_splits, tiles_per_split, n_stages;
+    int n_extra;      // key tiles of fresh rows attended by the last CTA of every cluster (0: nothing to refresh)
     int dl;           // output columns merged by one CTA of the cluster (even; the last CTA may own fewer)
     int q_tma;        // 1: the producer fetches Q with one TMA box (one query head per column); 0: softmax warps stage it
-    uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0
+    uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0;
+                                                    // off_list: the stale-key bits, 16 bytes per refreshed cache tile
     float scale_log2;
 };
 
@@ -124,10 +129,10 @@ struct KeysParams {
 struct alignas(16) KeysShared {
     uint32_t tmem;
     int abort_flag;
-    int n_mine;                                // entries of the refresh list
-    int pad;
+    int pad[2];
     int slow_flag[2][2];                       // [tile parity][warpgroup]: the softmax of that tile raised its references
-    uint32_t patch_mask[kMaxTiles / 32];       // bit j: tile j of this CTA holds a refreshed position
+    uint32_t patch_mask[kMaxTiles / 32];       // bit t: cache tile t of this CTA holds a refreshed (stale) position
+    uint16_t slot_base[kMaxTiles / 32];        // refreshed tiles before word w of the mask: tile -> row of the stale-key bits
     alignas(16) float m[kMaxSlots];            // reference maxima of the query rows, log2 units (read as float2)
     alignas(16) float factor[2][kMaxSlots];    // [tile parity]: rescale factors of that tile's slow path
     alignas(16) float lpart[2][kMaxSlots];     // row sums of the CTA's keys, one partial per group of row-sum threads
@@ -137,7 +142,9 @@ struct alignas(16) KeysShared {
 template <int N>
 __global__ void __launch_bounds__(64 + (N > 64 ? 256 : 128) + kAuxThreads, N <= 64 ? 2 : 1)
 attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                        const __grid_constant__ CUtensorMap map_q, const KeysParams p) {
+                        const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kn,
+                        const __grid_constant__ CUtensorMap map_vn, const __grid_constant__ CUtensorMap map_k1,
+                        const __grid_constant__ CUtensorMap map_v1, const KeysParams p) {
     static_assert(N == 48 || N == 64 || N == 96, "query-row slots per CTA");
     constexpr int WG = N > 64 ? 2 : 1;          // softmax warpgroups: each takes NH of a key's N scores
     constexpr int NH = N / WG;
@@ -155,7 +162,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const uint32_t bars = base + p.off_bar;
     KeysShared* sh = reinterpret_cast<KeysShared*>(gbase + p.off_bar + kBarBytes);
     volatile int* abort_flag = &sh->abort_flag;
-    int2* list = reinterpret_cast<int2*>(gbase + p.off_list);   // (active row i, position) pairs of this CTA's key range
+    uint32_t* stale = reinterpret_cast<uint32_t*>(gbase + p.off_list);   // [refreshed cache tile][4]: a bit per stale key
     auto bar = [&](int idx) { return bars + idx * 8; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -169,31 +176,38 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int n_tiles_total = (p.ctx_len + BK - 1) / BK;
     const int t_begin = split * p.tiles_per_split;
     const int t_end = min(n_tiles_total, t_begin + p.tiles_per_split);
-    const int T = t_end - t_begin;   // >= 1 by construction of the plan
+    const int TC = max(0, t_end - t_begin);                  // cache tiles of this CTA
     const int NS = p.n_stages;
     const bool refresh = p.k_new != nullptr;
+    // the last CTA of the cluster attends to the fresh rows first, as XT extra key tiles read from k_new / v_new
+    const int XT = (refresh && split == p.n_splits - 1) ? p.n_extra : 0;
+    const int T = XT + TC;           // tiles this CTA visits: >= 1 by construction of the plan
     const int key_lo = t_begin * BK, key_hi = min(p.ctx_len, t_end * BK);
     // exchange areas of the merge, from the start of the (then dead) Q / P^T / stage memory: C staging chunks (one per
-    // owner), C receive chunks (one per source), the weight table, the rows' output offsets.  A chunk holds
+    // owner), C receive chunks (one per source).  A chunk holds
     // [N queries][DL columns] floats of O^T, then m[N], then l[N].
     const uint32_t chunk_floats = (uint32_t)(N * DL + 2 * N);
     const uint32_t chunk_bytes = chunk_floats * 4u;
-    const uint32_t stg_off = 0, recv_off = (uint32_t)C * chunk_bytes, wgt_off = 2u * C * chunk_bytes,
-                   qoff_off = wgt_off + 8u * N * 4u;
+    const uint32_t stg_off = 0, recv_off = (uint32_t)C * chunk_bytes;
 
     // ---- set-up (touches no global memory) -------------------------------------------------
     if (tid == 0) {
         prefetch_map(&map_k);
         prefetch_map(&map_v);
         if (p.q_tma) prefetch_map(&map_q);
+        if (p.k_new) {
+            prefetch_map(&map_kn);
+            prefetch_map(&map_vn);
+            prefetch_map(&map_k1);
+            prefetch_map(&map_v1);
+        }
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1;
             if (i == B_PFULL || (i == B_QFULL && !p.q_tma)) count = kSoft;
-            if (i == B_PSUM || (i >= B_PATCHED && i < B_PATCHED + kMaxStages)) count = kAuxThreads;
+            if (i == B_PSUM || i == B_FRESHOUT || i == B_FRESHOUT + 1) count = kAuxThreads;
             mbar_init(bar(i), count);
         }
         sh->abort_flag = 0;
-        sh->n_mine = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (C > 1) mbar_expect_tx(bar(B_RECV), (uint32_t)C * chunk_bytes);   // the peers' partials, one chunk each
     }
@@ -221,16 +235,25 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             for (int j = 0; j < T; ++j) {
                 const int s = j % NS, u = j / NS;
                 if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
-                const int key0 = (t_begin + j) * BK;
+                if (u > 0 && j - NS < XT && sub == 0)   // the stage held a fresh tile: the cache update has read it
+                    mbar_wait(bar(B_FRESHOUT + (j - NS)), 0, abort_flag, p.dev_status);   // (one single-phase barrier per fresh tile)
                 const uint32_t dst = base + p.off_stage + s * STAGE;
                 mbar_expect_tx(bar(B_FULL + s), STAGE);
-                tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
-                tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
+                if (j < XT) {   // active rows [128 j, 128 j + 128) of this kv head, fresh; rows past n_active read as zero
+                    tma_load_5d(dst, &map_kn, 0, j * BK, 0, hk, b, bar(B_FULL + s));
+                    tma_load_5d(dst + TILE, &map_vn, 0, j * BK, 0, hk, b, bar(B_FULL + s));
+                } else {
+                    const int key0 = (t_begin + j - XT) * BK;
+                    tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
+                    tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
+                }
             }
         }
     } else if (warp == 1) {
-        // ================= refresh list, then MMA issue (lane 0) =================================
+        // ================= stale-key masks, then MMA issue (lane 0) =================================
         if (refresh) {
+            // which cached keys of this CTA's range are about to be refreshed: they are attended from k_new / v_new (as
+            // extra tiles, by the last CTA of the cluster), so their cached copies must not count
             int posv[kMaxActive / 32];
 #pragma unroll
             for (int k = 0; k < kMaxActive / 32; ++k) {
@@ -239,42 +262,47 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 if (k * 32 >= p.n_active) continue;   // uniform: nothing of the list left
                 if (i < p.n_active) posv[k] = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
             }
-            int n_mine = 0;
 #pragma unroll
             for (int k = 0; k < kMaxActive / 32; ++k) {
                 if (k * 32 >= p.n_active) break;
-                const bool hit = posv[k] >= key_lo && posv[k] < key_hi;
-                const unsigned mk = __ballot_sync(0xffffffffu, hit);
-                if (hit) {
-                    list[n_mine + __popc(mk & ((1u << lane) - 1u))] = make_int2(k * 32 + lane, posv[k]);
+                if (posv[k] >= key_lo && posv[k] < key_hi) {
                     const int tile = (posv[k] - key_lo) / BK;
                     atomicOr(&sh->patch_mask[tile >> 5], 1u << (tile & 31));
                 }
-                n_mine += __popc(mk);
             }
             __syncwarp();
-            if (lane == 0) {
-                sh->n_mine = n_mine;
-                mbar_arrive(bar(B_LIST));   // release: the list and the mask above are visible to whoever waits
+            {   // rows of the bit table: refreshed tiles in tile order (exclusive prefix count over the mask words)
+                const int cnt = __popc(sh->patch_mask[lane]);
+                int incl = cnt;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                sh->slot_base[lane] = (uint16_t)(incl - cnt);
+                const int total = __shfl_sync(0xffffffffu, incl, 31);
+                for (int w = lane; w < total * 4; w += 32) stale[w] = 0u;
             }
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < kMaxActive / 32; ++k) {
+                if (k * 32 >= p.n_active) break;
+                if (posv[k] >= key_lo && posv[k] < key_hi) {
+                    const int r = posv[k] - key_lo, tile = r / BK, kk = r % BK;
+                    const int slot = sh->slot_base[tile >> 5] + __popc(sh->patch_mask[tile >> 5] & ((1u << (tile & 31)) - 1u));
+                    atomicOr(&stale[slot * 4 + (kk >> 5)], 1u << (kk & 31));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_LIST));   // release: the masks above are visible to whoever waits
             __syncwarp();
         }
         if (lane == 0) {
             constexpr uint32_t IDESC_S = instr_desc2(N, 0, 0);    // A = K tile (K-major), B = Q (K-major)
             constexpr uint32_t IDESC_PV = instr_desc2(N, 1, 1);   // A = V tile (MN-major: d contiguous), B = P^T (MN-major)
             constexpr uint32_t QHALF = N * 128;                   // bytes of one 64-column half of the Q tile
-            // A tile that holds refreshed positions is handed to the patch warps once it has landed ("needs patch")
-            // and used once they are done ("patched"); one barrier pair per stage, and this thread waits for the
-            // answer before it goes on, so neither side can run a phase ahead of the other.
-            uint32_t n_patched = 0;   // bit s: parity of the patches of stage s so far
             auto issue_s = [&](int j) {
                 const int s = j % NS;
-                mbar_wait(bar(B_FULL + s), (j / NS) & 1, abort_flag, p.dev_status);
-                if (refresh && ((sh->patch_mask[j >> 5] >> (j & 31)) & 1u)) {
-                    mbar_arrive(bar(B_NEEDPATCH + s));
-                    mbar_wait(bar(B_PATCHED + s), (n_patched >> s) & 1u, abort_flag, p.dev_status);
-                    n_patched ^= 1u << s;
-                }
                 fence_after();
                 const uint32_t kst = base + p.off_stage + s * STAGE;
 #pragma unroll
@@ -285,77 +313,71 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 }
                 commit(bar(B_SFULL + (j & 1)));
             };
+            // S of tile j needs the tile (and its patch); P V of tile j needs P^T from the softmax.  Whichever is ready
+            // is issued: P V of a tile does not wait for the next tile to land (its commit frees the stage for the
+            // producer), S may run one tile ahead of P V (two S^T buffers).
             mbar_wait(bar(B_QFULL), 0, abort_flag, p.dev_status);
-            issue_s(0);
-            for (int j = 0; j < T; ++j) {
-                if (j + 1 < T) issue_s(j + 1);
-                const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + TILE;
-                mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
-                fence_after();
+            int next_s = 0, next_pv = 0;
+            SpinGuard guard;
+            while (next_pv < T) {
+                bool progressed = false;
+                if (next_s < T && next_s <= next_pv + 1 && mbar_try(bar(B_FULL + next_s % NS), (next_s / NS) & 1)) {
+                    issue_s(next_s);   // (the tile has landed)
+                    ++next_s;
+                    progressed = true;
+                }
+                if (mbar_try(bar(B_PFULL), next_pv & 1)) {
+                    const int j = next_pv;
+                    const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + TILE;
+                    fence_after();
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k)
-                    mma_ss(tmem + TM_O, smem_desc(vst + k * 2048, SUB, 1024), smem_desc(base + p.off_p + k * 2048, SUB, 1024),
-                           IDESC_PV, (j > 0 || k > 0));
-                commit(bar(B_PVDONE));
-                commit(bar(B_EMPTY + j % NS));
+                    for (int k = 0; k < BK / 16; ++k)
+                        mma_ss(tmem + TM_O, smem_desc(vst + k * 2048, SUB, 1024), smem_desc(base + p.off_p + k * 2048, SUB, 1024),
+                               IDESC_PV, (j > 0 || k > 0));
+                    commit(bar(B_PVDONE));
+                    commit(bar(B_EMPTY + j % NS));
+                    ++next_pv;
+                    progressed = true;
+                }
+                if (progressed) guard.progress();
+                else if (!guard.tick(abort_flag, p.dev_status)) break;
             }
         }
     } else if (warp >= 2 + 4 * WG) {
-        // ===== auxiliary warps: fresh rows over the landed tiles (and into the cache); row sums of P^T =====
+        // ===== auxiliary warps: the fresh rows into the cache (for later steps); row sums of P^T =====
         const int atid = tid - (64 + kSoft);
-        int n_mine = 0;
-        if (refresh) {
-            mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
-            n_mine = sh->n_mine;
+        if (XT > 0 && sub == 0) {
+            // One CTA per (sequence, kv head) -- the one that attends to the fresh tiles -- also puts the active rows'
+            // K/V into the cache, for later steps: the fresh tile is in shared memory already, so each row leaves as four
+            // TMA stores of 128 bytes (K and V, two 64-column halves) to its position in the cache.  Nothing in this launch
+            // depends on these stores; the producer only waits until they have read the tile before it refills the stage.
+            int posx[2];
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {   // positions of this thread's rows of the first fresh tile, fetched ahead
+                const int i = rr * kAuxThreads + atid;
+                posx[rr] = (i < p.n_active) ? (p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i) : -1;
+            }
+            for (int x = 0; x < XT; ++x) {
+                mbar_wait(bar(B_FULL + x % NS), (x / NS) & 1, abort_flag, p.dev_status);   // the fresh tile has landed
+                const uint32_t tile = base + p.off_stage + (x % NS) * STAGE;
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int r = rr * kAuxThreads + atid, i = x * BK + r;
+                    int pos = posx[rr];
+                    if (x > 0) pos = (i < p.n_active) ? (p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i) : -1;
+                    if (pos >= 0 && pos < p.ctx_len) {
+                        const uint32_t row = tile + (r >> 3) * 1024 + (r & 7) * 128;
+                        tma_store_4d(&map_k1, 0, pos, 0, bh, row);
+                        tma_store_4d(&map_k1, 0, pos, 1, bh, row + SUB);
+                        tma_store_4d(&map_v1, 0, pos, 0, bh, row + TILE);
+                        tma_store_4d(&map_v1, 0, pos, 1, bh, row + TILE + SUB);
+                    }
+                }
+                bulk_commit();
+                bulk_wait_read();
+                mbar_arrive(bar(B_FRESHOUT + x));
+            }
         }
-        const bool writer = sub == 0;   // one CTA column per kv head updates the cache in global memory
-        // 16-byte pieces of the list's rows that fall into tile j: entry e = c >> 5, K pieces 0..15 then V pieces 0..15.
-        // A thread holds up to kPatchPer pieces of one round in registers, so the loads of a tile's fresh rows are in
-        // flight while the tile itself is still landing.
-        uint4 pv[kPatchPer];
-        auto patch_loads = [&](int j, int round) {
-            const int key0 = key_lo + j * BK;
-#pragma unroll
-            for (int u = 0; u < kPatchPer; ++u) {
-                const int c = (round * kPatchPer + u) * kAuxThreads + atid;
-                if (c < n_mine * 32) {
-                    const int2 ip = list[c >> 5];
-                    if (ip.y >= key0 && ip.y < key0 + BK) {
-                        const long long src = (((long long)b * p.n_active + ip.x) * p.n_kv_heads + hk) * HD + (c & 15) * 8;
-                        pv[u] = __ldg(reinterpret_cast<const uint4*>(((c & 16) ? p.v_new : p.k_new) + src));
-                    }
-                }
-            }
-        };
-        auto patch_stores = [&](int j, int round) {
-            const int key0 = key_lo + j * BK;
-            unsigned char* kt = gbase + p.off_stage + (j % NS) * STAGE;
-#pragma unroll
-            for (int u = 0; u < kPatchPer; ++u) {
-                const int c = (round * kPatchPer + u) * kAuxThreads + atid;
-                if (c < n_mine * 32) {
-                    const int2 ip = list[c >> 5];
-                    if (ip.y >= key0 && ip.y < key0 + BK) {
-                        const int r = ip.y - key0, piece = c & 15, isv = (c >> 4) & 1;
-                        const uint32_t off = (uint32_t)isv * TILE + (uint32_t)(piece >> 3) * SUB + (r >> 3) * 1024 + (r & 7) * 128 +
-                                             (((piece & 7) ^ (r & 7)) << 4);
-                        *reinterpret_cast<uint4*>(kt + off) = pv[u];
-                        if (writer)
-                            *reinterpret_cast<uint4*>((isv ? p.v_cache : p.k_cache) + ((long long)bh * p.ctx_len + ip.y) * HD + piece * 8) =
-                                pv[u];
-                    }
-                }
-            }
-        };
-        auto next_patched = [&](int from) {   // first tile >= from that holds a refreshed position (T if none)
-            for (int j = from; j < T; ++j)
-                if ((sh->patch_mask[j >> 5] >> (j & 31)) & 1u) return j;
-            return T;
-        };
-        const int n_rounds = (n_mine * 32 + kPatchPer * kAuxThreads - 1) / (kPatchPer * kAuxThreads);
-        int np = n_mine > 0 ? next_patched(0) : T;
-        if (np < T) patch_loads(np, 0);
-        uint32_t n_needed = 0;   // bit s: parity of the "needs patch" hand-overs of stage s so far
 
         // row sums: this thread adds up column pair cp of the keys [k_lo, k_lo + BK / kParts) of every tile
         const bool summer = atid < kPairs * kParts;
@@ -365,20 +387,6 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         float acc0 = 0.f, acc1 = 0.f;
 
         for (int j = 0; j < T; ++j) {
-            // every tile up to j + 1 that needs its fresh rows gets them now: S of tile j + 1 is issued before P V of tile j
-            while (np <= j + 1 && np < T) {
-                const int s = np % NS;
-                mbar_wait(bar(B_NEEDPATCH + s), (n_needed >> s) & 1u, abort_flag, p.dev_status);   // the tile has landed
-                n_needed ^= 1u << s;
-                for (int round = 0; round < n_rounds; ++round) {
-                    if (round > 0) patch_loads(np, round);
-                    patch_stores(np, round);
-                }
-                fence_async_smem();     // patched rows (generic proxy) -> visible to the tensor core (async proxy)
-                mbar_arrive(bar(B_PATCHED + s));
-                np = next_patched(np + 1);
-                if (np < T) patch_loads(np, 0);
-            }
             // P^T of tile j is in shared memory
             mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
             if (summer) {
@@ -435,12 +443,38 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         // P^T row of this key: [64-slot half][key][64 slots], 128-byte swizzle
         unsigned char* prow = gbase + p.off_p + (kk >> 3) * 1024 + (kk & 7) * 128;
         const int bar_or = 2 + 2 * wg, bar_sync = 3 + 2 * wg;   // named barriers of this warpgroup
+        // which keys of the fresh tiles exist: active rows with a position inside the context (bit x: row 128 x + kk)
+        uint32_t fresh_ok = 0;
+        for (int x = 0; x < XT; ++x) {
+            const int i = x * BK + kk;
+            if (i < p.n_active) {
+                const int pos = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
+                if (pos >= 0 && pos < p.ctx_len) fresh_ok |= 1u << x;
+            }
+        }
+        bool masks_ready = !refresh;   // the stale-key bits are awaited once, before the first cache tile
 
         for (int j = 0; j < T; ++j) {
             mbar_wait(bar(B_SFULL + (j & 1)), (j >> 1) & 1, abort_flag, p.dev_status);
             fence_after();
             const uint32_t s_addr = tmem + lane_addr + TM_S + (j & 1) * NP + c0;
-            const bool past_end = (t_begin + j) * BK + kk >= p.ctx_len;   // only in the ragged last tile of the context
+            // this thread's key does not count: a missing row of a fresh tile, a key past the end of the context (ragged
+            // last tile), a cached key whose position is being refreshed (it is attended from the fresh tile instead)
+            bool past_end;
+            if (j < XT) {
+                past_end = !((fresh_ok >> j) & 1u);
+            } else {
+                const int t = j - XT;
+                past_end = (t_begin + t) * BK + kk >= p.ctx_len;
+                if (!masks_ready) {
+                    mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
+                    masks_ready = true;
+                }
+                if (refresh && ((sh->patch_mask[t >> 5] >> (t & 31)) & 1u)) {
+                    const int slot = sh->slot_base[t >> 5] + __popc(sh->patch_mask[t >> 5] & ((1u << (t & 31)) - 1u));
+                    past_end = past_end || ((stale[slot * 4 + (kk >> 5)] >> (kk & 31)) & 1u);
+                }
+            }
             // d = s * scale * log2(e) - m[q]; does any score exceed its reference by more than 2^8?
             f32x2 d2[NH / 2];
             auto load_d = [&]() {
@@ -523,8 +557,9 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         fence_after();
         if (C > 1) {
             // first cluster barrier, arrive half: the peers may write their partials into this CTA's receive chunks
+            // (nothing is published by it, so no memory ordering is attached)
             __syncwarp();
-            cluster_arrive();
+            cluster_arrive_relaxed();
         }
         mbar_wait(bar(B_PSUM), (T - 1) & 1, abort_flag, p.dev_status);     // the row sums are complete
 
@@ -574,7 +609,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     if (C > 1) {
         if (!(warp >= 2 && warp < 2 + 4 * WG)) {   // the other warps' halves of the first cluster barrier
             __syncwarp();
-            cluster_arrive();
+            cluster_arrive_relaxed();
             cluster_wait();
         }
         // ---- merge the C partials of the output columns this CTA owns -------------------------
@@ -582,48 +617,42 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         // second cluster barrier, arrive half: this CTA holds every peer's partial, so the peers' copies out of their
         // staging chunks have completed; the wait half, before leaving, overlaps the merge
         __syncwarp();
-        cluster_arrive();
+        cluster_arrive_relaxed();
         const float* recv = reinterpret_cast<const float*>(gbase + recv_off);
-        float* wgt = reinterpret_cast<float*>(gbase + wgt_off);                  // [8][N] weights 2^(m_s - m) / l
-        long long* qoff = reinterpret_cast<long long*>(gbase + qoff_off);        // [N] element offset of each query row in out
-        // weights: eight lanes per query row, one per source
-        for (int it0 = 0; it0 < rows_total * 8; it0 += kThreads) {
-            const int it = it0 + tid, q = it >> 3, s = it & 7;
-            const bool live = q < rows_total && s < C;
-            const float ms = live ? recv[s * chunk_floats + N * DL + q] : -INFINITY;
-            const float ls = live ? recv[s * chunk_floats + N * DL + N + q] : 0.f;
-            float m = ms;
-            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
-            const float e = live ? fast_exp2(ms - m) : 0.f;
-            float l = e * ls;
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
-            l += __shfl_xor_sync(0xffffffffu, l, 4);
-            if (live) wgt[s * N + q] = e / l;
-        }
-        if (tid < rows_total) {
-            const int i = i0 + tid / p.group, jh = tid % p.group;
-            qoff[tid] = (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL;
-        }
-        __syncthreads();
-        // a thread owns two adjacent output columns of a query row: one 4-byte store
+        // a thread owns two adjacent output columns of a query row (one 4-byte store) and works out the row's weights
+        // 2^(m_s - m) / l itself: the sixteen or so threads of a row repeat that, but nobody waits for a table
         const int half_dl = min(DL, HD - split * DL) / 2;
         if (!*abort_flag) {
             for (int idx = tid; idx < rows_total * half_dl; idx += kThreads) {
                 const int qq = idx / half_dl, dp = idx % half_dl;
-                float a0 = 0.f, a1 = 0.f;
+                float ms[8], ls[8];
+                float2 v[8];
 #pragma unroll
                 for (int s = 0; s < 8; ++s) {
                     if (s < C) {
-                        const float w = wgt[s * N + qq];
-                        const float2 v = *reinterpret_cast<const float2*>(recv + s * chunk_floats + qq * DL + 2 * dp);
-                        a0 = fmaf(w, v.x, a0);
-                        a1 = fmaf(w, v.y, a1);
+                        const float* ch = recv + s * chunk_floats;
+                        ms[s] = ch[N * DL + qq];
+                        ls[s] = ch[N * DL + N + qq];
+                        v[s] = *reinterpret_cast<const float2*>(ch + qq * DL + 2 * dp);
+                    } else {
+                        ms[s] = -INFINITY;
+                        ls[s] = 0.f;
+                        v[s] = make_float2(0.f, 0.f);
                     }
                 }
-                *reinterpret_cast<uint32_t*>(p.out + qoff[qq] + 2 * dp) = pack_bf16x2(a0, a1);
+                const float m = fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
+                float l = 0.f, a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    const float e = fast_exp2(ms[s] - m);   // 0 for the sources that do not exist
+                    l = fmaf(e, ls[s], l);
+                    a0 = fmaf(e, v[s].x, a0);
+                    a1 = fmaf(e, v[s].y, a1);
+                }
+                const float inv = 1.f / l;
+                const int i = i0 + qq / p.group, jh = qq % p.group;
+                __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL + 2 * dp;
+                *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(a0 * inv, a1 * inv);
             }
         }
         // no CTA leaves while a peer may still copy out of its staging chunks
@@ -654,6 +683,20 @@ bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// the same cache as the target of the refresh: boxes of one key and one 64-column half (128 bytes), so that a row of a
+// tile in shared memory can be stored to an arbitrary position
+bool make_cache_row_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {64, (cuuint64_t)ctx_len, 2, (cuuint64_t)bh};
+    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)ctx_len * HD * 2};
+    const cuuint32_t box[4] = {64, 1, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(cache), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // q [B, n, H_q, 128] bf16 (one query head per CTA column) seen as 5-D {64 columns, row, head, half, sequence}:
 // the box {64, N, 1, 2, 1} lands as [half][row][64 columns], the K-major Q tile; rows past n read as zero
 bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_q_heads, int n_slots) {
@@ -672,7 +715,7 @@ bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_
 struct KeysPlan {
     bool ok;
     int group, rows_chunk, n_sub_r, n_sub;   // heads and active rows per CTA column, row chunks, CTA columns per kv head
-    int n_slots, n_splits, tiles_per_split, n_stages, dl, ctas_per_sm;
+    int n_slots, n_splits, tiles_per_split, n_stages, n_extra, dl, ctas_per_sm;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
 };
 
@@ -682,8 +725,9 @@ constexpr uint32_t kSmemTwoPerSm = 115712;   // (228 KB per SM - 2 x 1 KB reserv
 // tensor-memory columns the instantiation for n_slots allocates (see TM_COLS in the kernel)
 constexpr int tm_columns(int n_slots) { return 3 * (n_slots <= 64 ? 64 : 128) <= 256 ? 256 : 512; }
 
-// shared-memory carve for n_slots query slots and ns stages
-void carve(KeysPlan& pl, int n_active, int ns) {
+// shared-memory carve for n_slots query slots and ns stages; `fresh`: room for the stale-key bits (16 bytes per
+// refreshed cache tile, of which there are at most n_active)
+void carve(KeysPlan& pl, int n_active, int ns, bool fresh) {
     uint32_t off = (uint32_t)pl.n_slots * 256u;   // Q
     off = (off + 1023u) & ~1023u;
     pl.off_p = off;
@@ -691,7 +735,7 @@ void carve(KeysPlan& pl, int n_active, int ns) {
     pl.off_stage = off;
     off += (uint32_t)ns * STAGE;
     pl.off_list = off;
-    off += ((uint32_t)n_active * 8u + 15u) & ~15u;
+    off += fresh ? (uint32_t)n_active * 16u : 0u;
     pl.off_bar = off;
     off += kBarBytes + (uint32_t)sizeof(KeysShared) + 16u;
     pl.smem_bytes = off + 1024u;
@@ -702,7 +746,55 @@ void carve(KeysPlan& pl, int n_active, int ns) {
     pl.n_stages = ns;
 }
 
-KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
+// How many clusters of c CTAs with this much dynamic shared memory the current device keeps resident at once (clusters
+// are placed inside one GPC, so this can be fewer than SMs x CTAs per SM / c); -1 when it cannot be asked (no device).
+// Asked once per (device, instantiation, cluster size, shared memory) and remembered.
+template <int N>
+int resident_clusters_of(int c, uint32_t smem) {
+    static PerDeviceOnce attr_once;
+    if (ensure_dynamic_smem(attr_once, attend_skip_keys_kernel<N>, (int)kSmemMax) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(c, 1, 1);
+    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + kAuxThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = c;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, attend_skip_keys_kernel<N>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    return n;
+}
+
+int resident_clusters(int n_slots, int c, uint32_t smem) {
+    struct Entry { int dev, n_slots, c; uint32_t smem; int clusters; };
+    static std::mutex mu;
+    static std::vector<Entry> seen;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : seen)
+        if (e.dev == dev && e.n_slots == n_slots && e.c == c && e.smem == smem) return e.clusters;
+    const int n = n_slots == 48 ? resident_clusters_of<48>(c, smem) : n_slots == 64 ? resident_clusters_of<64>(c, smem)
+                                                                                      : resident_clusters_of<96>(c, smem);
+    seen.push_back({dev, n_slots, c, smem, n});
+    return n;
+}
+
+// fresh: the call refreshes (k_new / v_new given), so the last CTA of every cluster also visits the fresh tiles
+KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active, bool fresh) {
     KeysPlan pl{};
     // a CTA column takes the largest divisor of the H_q / H_kv heads of a kv head whose packed rows fit the query
     // slots; the other columns of that kv head stream the same K/V (from L2) for their own heads
@@ -716,48 +808,79 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active) {
     pl.n_sub = (g / pl.group) * pl.n_sub_r;
     const int rows = pl.rows_chunk * pl.group;
     pl.n_slots = rows <= 48 ? 48 : rows <= 64 ? 64 : 96;
+    pl.n_extra = fresh ? (n_active + BK - 1) / BK : 0;
     const int tm_cols = tm_columns(pl.n_slots);
     const int key_tiles = (d.ctx_len + BK - 1) / BK;
     const long long columns = (long long)d.batch * d.n_kv_heads * pl.n_sub;   // grid.y
     const int sms = sm_count();
-    // cluster size: every CTA at least one tile, all CTAs resident at once (two per SM when they are small), and
-    // the most-loaded SM streaming as few tiles as possible; among equals, more CTAs (more SMs pulling)
-    long long best_load = -1, best_ctas = 0;
-    for (int c = 1; c <= 8 && c <= key_tiles; ++c) {
-        const int tps = (key_tiles + c - 1) / c;
-        if ((key_tiles + tps - 1) / tps != c || tps > kMaxTiles) continue;   // this c leaves a CTA empty
-        int dl = (HD + c - 1) / c;
-        dl += dl & 1;
-        if ((c - 1) * dl >= HD) continue;                                    // an owner without columns
-        KeysPlan t = pl;
-        int ns = tps < kMaxStages ? tps : kMaxStages;
-        carve(t, n_active, ns);
-        while (ns > 1 && t.smem_bytes > kSmemMax) carve(t, n_active, --ns);
-        if (t.smem_bytes > kSmemMax || (ns < 2 && tps > 1)) continue;
-        // the exchange areas of the merge (2 c chunks, weights, row offsets) reuse the Q / P^T / stage memory
-        if (c > 1 && 2 * (size_t)c * (pl.n_slots * dl + 2 * pl.n_slots) * 4 + (size_t)pl.n_slots * 40 > t.off_list) continue;
-        const int per_sm = (t.smem_bytes <= kSmemTwoPerSm && tm_cols <= 256) ? 2 : 1;
-        const long long ctas = columns * c;
-        if (ctas > (long long)per_sm * sms) continue;
-        const long long load = (long long)tps * ((ctas + sms - 1) / sms);
-        if (best_load < 0 || load < best_load || (load == best_load && ctas > best_ctas)) {
-            best_load = load;
-            best_ctas = ctas;
-            pl.n_splits = c;
-            pl.tiles_per_split = tps;
-            pl.dl = dl;
-            pl.ctas_per_sm = per_sm;
-            pl.n_stages = ns;
+    // Cluster shape: cs CTAs split the cache tiles (every one at least one tile); the fresh tiles go to the last of
+    // them, or to one more CTA of their own (worth it when a CTA holds so few tiles that one more would be felt, and
+    // needed when it has a single stage).  All CTAs resident at once (two per SM when they are small); the most-loaded SM
+    // streams as few tiles as possible; among equals, more CTAs (more SMs pulling).
+    long long best_cost = -1, best_ctas = 0;
+    for (int cs = 1; cs <= 8 && cs <= key_tiles; ++cs) {
+        const int tps = (key_tiles + cs - 1) / cs;
+        if ((key_tiles + tps - 1) / tps != cs || tps > kMaxTiles) continue;   // this cs leaves a CTA empty
+        for (int own = 0; own <= (fresh ? 1 : 0); ++own) {                     // own: the fresh tiles get their own CTA
+            const int c = cs + own;
+            if (c > 8) continue;
+            int dl = (HD + c - 1) / c;
+            dl += dl & 1;
+            if ((c - 1) * dl >= HD) continue;                                  // an owner without columns
+            const int last_tiles = key_tiles - (cs - 1) * tps;
+            const int visits = own ? (tps > pl.n_extra ? tps : pl.n_extra)
+                                   : (tps > last_tiles + pl.n_extra ? tps : last_tiles + pl.n_extra);
+            KeysPlan t = pl;
+            int ns = visits < kMaxStages ? visits : kMaxStages;
+            carve(t, n_active, ns, fresh);
+            while (ns > 1 && t.smem_bytes > kSmemMax) carve(t, n_active, --ns, fresh);
+            if (t.smem_bytes > kSmemMax || (ns < 2 && visits > 1)) continue;
+            // the exchange areas of the merge (2 c chunks) reuse the Q / P^T / stage memory
+            if (c > 1 && 2 * (size_t)c * (pl.n_slots * dl + 2 * pl.n_slots) * 4 > t.off_list) continue;
+            const int per_sm = (t.smem_bytes <= kSmemTwoPerSm && tm_cols <= 256) ? 2 : 1;
+            const long long ctas = columns * c;
+            if (ctas > (long long)per_sm * sms) continue;
+            const int fit = resident_clusters(pl.n_slots, c, t.smem_bytes);   // (-1: no device to ask, keep the estimate)
+            if (fit >= 0 && columns > fit) continue;
+            // cost in quarter tiles: the fresh tiles arrive early (they are small and mostly in L2), so on a shared CTA
+            // they count a quarter of a cache tile
+            const long long cost = 4LL * tps * ((ctas + sms - 1) / sms) + ((fresh && !own) ? pl.n_extra : 0);
+            if (best_cost < 0 || cost < best_cost || (cost == best_cost && ctas > best_ctas)) {
+                best_cost = cost;
+                best_ctas = ctas;
+                pl.n_splits = c;
+                pl.tiles_per_split = tps;
+                pl.dl = dl;
+                pl.ctas_per_sm = per_sm;
+                pl.n_stages = ns;
+            }
         }
     }
-    pl.ok = best_load >= 0;
-    if (pl.ok) carve(pl, n_active, pl.n_stages);
+    pl.ok = best_cost >= 0;
+    if (pl.ok) carve(pl, n_active, pl.n_stages, fresh);
     return pl;
+}
+
+// k_new / v_new [B, n, H_kv, 128] bf16 seen as 5-D {64 columns, active row, half, kv head, sequence}: one box
+// {64, 128, 2, 1, 1} lands as [half][row][64 columns], i.e. exactly like a cache tile whose keys are the active rows
+// 128 j .. 128 j + 127 of one kv head; rows past n read as zero
+bool make_fresh_map(CUtensorMap* map, const void* fresh, int batch, int n_active, int n_kv_heads) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[5] = {64, (cuuint64_t)n_active, 2, (cuuint64_t)n_kv_heads, (cuuint64_t)batch};
+    const cuuint64_t strides[4] = {(cuuint64_t)n_kv_heads * HD * 2, 128, (cuuint64_t)HD * 2,
+                                   (cuuint64_t)n_active * n_kv_heads * HD * 2};
+    const cuuint32_t box[5] = {64, (cuuint32_t)BK, 2, 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(fresh), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int N>
 cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv,
-                     const CUtensorMap& mq, int bh, cudaStream_t stream) {
+                     const CUtensorMap& mq, const CUtensorMap& mkn, const CUtensorMap& mvn, const CUtensorMap& mk1,
+                     const CUtensorMap& mv1, int bh, cudaStream_t stream) {
     static PerDeviceOnce attr_once;
     if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_skip_keys_kernel<N>, (int)kSmemMax); ea != cudaSuccess)
         return ea;
@@ -775,40 +898,46 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, mq, p);
+    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, mq, mkn, mvn, mk1, mv1, p);
 }
 
 }  // namespace
 
-bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active) {
+bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active, bool fresh) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
     if (n_active > kMaxActive) return false;
-    const KeysPlan pl = make_keys_plan(d, n_active);
-    if (!pl.ok) return false;   // no cluster size keeps all CTAs resident: the row-major skip kernel streams better
+    const KeysPlan pl = make_keys_plan(d, n_active, fresh);
+    if (!pl.ok) return false;   // no cluster shape keeps all CTAs resident: the row-major skip kernel streams better
     if ((long long)d.batch * d.n_kv_heads * pl.n_sub > 65535) return false;   // grid.y
     // row chunks re-read the K/V of a head once per chunk: only worth it while the keys can still be split
     if (pl.n_sub_r > 1 && pl.n_splits < 2) return false;
     return true;
 }
 
-void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
-    const KeysPlan pl = make_keys_plan(d, n_active);
-    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u ctas_per_sm=%d", pl.n_slots,
-             pl.n_splits, d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes, pl.ctas_per_sm);
+void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, bool fresh, char* buf, size_t len) {
+    const KeysPlan pl = make_keys_plan(d, n_active, fresh);
+    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u ctas_per_sm=%d fresh_tiles=%d",
+             pl.n_slots, pl.n_splits, d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes, pl.ctas_per_sm,
+             pl.n_extra);
 }
 
 cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                     cudaStream_t stream) {
-    const KeysPlan pl = make_keys_plan(a.d, a.n_active);
+    const bool fresh = k_new != nullptr;
+    const KeysPlan pl = make_keys_plan(a.d, a.n_active, fresh);
     if (!pl.ok) return cudaErrorInvalidConfiguration;
     const int bh = a.d.batch * a.d.n_kv_heads;
     CUtensorMap map_k, map_v;
     if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
         return cudaErrorInvalidValue;
     KeysParams p{};
-    CUtensorMap map_q = map_k;   // unused unless q_tma
+    CUtensorMap map_q = map_k, map_kn = map_k, map_vn = map_v, map_k1 = map_k, map_v1 = map_v;   // placeholders unless q_tma / fresh
     p.q_tma = (pl.group == 1) ? 1 : 0;   // one query head per CTA column: its rows are one TMA box
     if (p.q_tma && !make_q_map(&map_q, a.q, a.d.batch, a.n_active, a.d.n_q_heads, pl.n_slots)) return cudaErrorInvalidValue;
+    if (fresh && (!make_fresh_map(&map_kn, k_new, a.d.batch, a.n_active, a.d.n_kv_heads) ||
+                  !make_fresh_map(&map_vn, v_new, a.d.batch, a.n_active, a.d.n_kv_heads) ||
+                  !make_cache_row_map(&map_k1, a.k_cache, bh, a.d.ctx_len) || !make_cache_row_map(&map_v1, a.v_cache, bh, a.d.ctx_len)))
+        return cudaErrorInvalidValue;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
     p.v_new = static_cast<const __nv_bfloat16*>(v_new);
@@ -828,6 +957,7 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.n_splits = pl.n_splits;
     p.tiles_per_split = pl.tiles_per_split;
     p.n_stages = pl.n_stages;
+    p.n_extra = pl.n_extra;
     p.dl = pl.dl;
     p.off_p = pl.off_p;
     p.off_stage = pl.off_stage;
@@ -835,9 +965,9 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
     const int cols = bh * pl.n_sub;
-    return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, cols, stream)
-           : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, cols, stream)
-                              : launch_n<96>(pl, p, map_k, map_v, map_q, cols, stream);
+    return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)
+           : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)
+                              : launch_n<96>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream);
 }
 
 }  // namespace ec

@@ -125,12 +125,12 @@ bool attend_skip_supported(const ec_attn_desc& d, int n_active);
 // host-only descriptions of the launch the plan functions choose ("kernel<instantiation> grid=... cluster=..."),
 // written into buf (always terminated)
 void attend_skip_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
-void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
+void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, bool fresh, char* buf, size_t len);
 void attend_dense_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len);
 cudaError_t launch_attend_skip(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                cudaStream_t stream);
 // skip-step path with the keys on the M axis (bf16, head_dim 128, n_active * H_q/H_kv <= 64)
-bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active);
+bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active, bool fresh);   // fresh: k_new / v_new are given
 cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, const void* v_new, const int32_t* active_idx,
                                     cudaStream_t stream);
 // two-row-tile dense path (bf16, head_dim 128): used when its (row-tile pair, kv head) units fill the GPU

@@ -57,6 +57,31 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     if (dev_status) atomicExch(dev_status, (int)EC_ERR_TIMEOUT);
 }
+// bookkeeping of a bounded polling loop over several barriers (same limits as mbar_wait): call tick() after a round
+// without progress; it returns false when the loop should give up (limit reached: abort raised; or abort already set)
+struct SpinGuard {
+    uint32_t n = 0;
+    unsigned long long t0 = 0;
+    __device__ __forceinline__ bool tick(volatile int* abort_flag, int32_t* dev_status) {
+        if ((++n & 63u) != 0) return true;
+        if (*abort_flag) return false;
+        const unsigned long long now = global_timer_ns();
+        if (t0 == 0) t0 = now;
+        if (n < kSpinLimit && now - t0 <= kWaitLimitNs) return true;
+        *abort_flag = 1;
+        if (dev_status) atomicExch(dev_status, (int)EC_ERR_TIMEOUT);
+        return false;
+    }
+    __device__ __forceinline__ void progress() { n = 0; t0 = 0; }
+};
+// 16-byte read-only load issued exactly here when `pred` holds (the destination keeps its value otherwise): the
+// compiler can neither move it nor turn it into a load followed by a select that would wait for the data
+__device__ __forceinline__ void ldg_nc_v4_pred(uint4& v, const void* ptr, bool pred) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "@p ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];\n\t}"
+        : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "l"(ptr), "r"((uint32_t)pred) : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
@@ -67,6 +92,13 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
 }
+// TMA store of one box from shared memory (bulk async-group completion)
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int x, int y, int z, int w, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_map(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -160,6 +192,8 @@ __host__ __device__ constexpr uint32_t instr_desc2(int n, int a_mn, int b_mn) {
 }
 // cluster helpers
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// arrive half without memory ordering: for barriers that only say "this CTA has got this far"
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t cta_rank) {
     uint32_t r;
