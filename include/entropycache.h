@@ -139,7 +139,10 @@ size_t ec_entropy_gate_workspace_bytes(int32_t n_rows, int32_t vocab);
  * logits: [n_rows, row_stride_elems] of `dtype`, only the first `vocab` columns of
  * a row are read; -inf entries are allowed (probability 0), +inf/NaN are not.
  * argmax_out / conf_out / entropy_out may each be NULL.  n_rows must be a
- * multiple of rows_per_seq.  Arithmetic is fp32.  workspace as for ec_attend. */
+ * multiple of rows_per_seq.  Arithmetic is fp32.  workspace as for ec_attend.
+ * The kernel's waits on its own staged copies are bounded (one second); should one ever give up, the sequences
+ * it touched get decision_out[b] = -1 (neither EC_SKIP nor EC_RECOMPUTE) and unspecified per-row outputs, and the
+ * workspace stays reusable.  The same holds for the other gate entry points below. */
 ec_status ec_entropy_gate(const void *logits, int32_t dtype, int32_t n_rows, int32_t vocab,
                           int64_t row_stride_elems, int32_t rows_per_seq,
                           const uint8_t *decoded_flags, float tau,

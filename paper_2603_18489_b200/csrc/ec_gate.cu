@@ -3,12 +3,15 @@
 // entropy over the rows flagged "newly decoded" and its comparison with tau
 // (Algorithm 1: E > tau -> recompute, else skip).
 //
-// The pass is HBM-bound: R*V*sizeof(elem) bytes are read exactly once; the arithmetic is kept to about
-// six instructions per element so that the issue slots do not become the limit first.
+// R*V*sizeof(elem) bytes are read exactly once; the arithmetic is about seven instructions per element.
 //   grid  = (splits, R): CTA (s, r) owns the columns [s*chunk, (s+1)*chunk) of row r; the split count is
-//           chosen so that the whole grid is about one resident wave (4 CTAs of 256 threads per SM);
-//   loop  : a thread visits its columns in ascending order, four 16-byte vectors (bf16x8 / f32x4) per
-//           iteration, the next four already in flight (register double buffer), and keeps a running
+//           chosen so that the whole grid is about one resident wave (4 CTAs per SM);
+//   CTA   : 8 consumer warps and one producer warp.  The producer's lane 0 moves the chunk through a ring of
+//           three 16 KB stages in shared memory with bulk copies (cp.async.bulk, completion on an mbarrier, L2
+//           evict-first), as far ahead as the ring allows, so the bytes in flight per SM are the rings of its
+//           resident CTAs and do not depend on the consumers' registers;
+//   loop  : a consumer thread takes the 16-byte vectors (bf16x8 / f32x4) t, t + 256, ... of the chunk in ascending
+//           order, four per stage, and keeps a running
 //           (max, S, T) with S = sum 2^d, T = sum 2^d * d, d = x*log2(e) - base: one ex2.approx per element
 //           and one packed fp32x2 FMA, add and FMA per pair of elements.  The base follows the maximum lazily: it moves, and S and T
 //           are rescaled (S' = 2^dl S, T' = 2^dl (T + dl S), dl = old base - new base), only when a value
@@ -18,7 +21,7 @@
 //   argmax: the thread remembers the iteration that raised its maximum; after the CTA-wide maximum is
 //           known, only the threads that attained it look at that iteration's vectors again for the
 //           first column (ties -> smallest index, through every reduction stage);
-//   CTA   : sums rescaled to the CTA's base and added (shuffles + shared memory);
+//   reduce: sums rescaled to the CTA's base and added (shuffles + shared memory);
 //   merge : CTA partial (M, S, T, idx) -> workspace, one atomic ticket; the last CTA of a sequence
 //           (no spinning: tickets only count arrivals) merges the partials of every row of the
 //           sequence, writes H = ln S - ln2 * T / S, conf = 2^(M*log2e - base) / S and argmax, takes
@@ -27,19 +30,26 @@
 // The entropy identity used: with p_j = 2^{d_j} / S,  -sum p_j ln p_j = ln S - ln2 * T / S
 // for any common base, so no partial ever needs the true row maximum.
 // The kernel is launched with programmatic stream serialisation and touches global memory only after
-// griddepcontrol.wait.
+// griddepcontrol.wait.  Every mbarrier wait is bounded (one second); a CTA whose wait gave up waits, bounded
+// again, for its copies in flight, still arrives at its ticket with a poison bit, and the sequence then reports
+// decision -1 instead of a value computed from missing data.
 #include "ec_common.cuh"
+#include "ec_tc_ptx.cuh"
 
 #include <float.h>
 
 namespace ec {
 namespace {
 
-constexpr int kGateThreads = 256;
+constexpr int kGateThreads = 256;      // consumer threads of a CTA (a producer warp comes on top)
+constexpr int kCtasPerSm = 4;
 constexpr int kVec = 8;  // columns per thread in one slab of kGateThreads * kVec columns (chunk granularity)
 constexpr int kMaxSplits = 96;
 constexpr float kDClamp = -150.0f;  // 2^-150 flushes to 0 (ftz)
-constexpr int kUnroll = 4;          // 16-byte vectors per thread per iteration
+constexpr int kStages = 3;                          // ring of staged buffers per CTA
+constexpr int kStageVecs = 4 * kGateThreads;        // 16-byte vectors per stage: four per consumer thread
+constexpr uint32_t kStageBytes = kStageVecs * 16u;
+constexpr int kPoison = 1 << 20;                    // added to a ticket by a CTA whose wait gave up
 constexpr int kSingleLevelMaxRows = 64;
 constexpr float kRebase = 64.f;     // the base moves when a value exceeds it by more than 2^kRebase
 constexpr unsigned int kXMinBf16x2 = 0xFE96FE96u;   // two bf16 of about -1e38: lower clamp of the logits
@@ -94,6 +104,23 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// global -> shared bulk copy that completes on an mbarrier; the source is read once, so it leaves L2 first
+__device__ __forceinline__ uint64_t evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// barrier of the 256 consumer threads (the producer warp leaves early)
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kGateThreads) : "memory"); }
 __device__ __forceinline__ unsigned int max_bf16x2(unsigned int a, unsigned int b) {
     unsigned int d;
     asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
@@ -223,7 +250,7 @@ __device__ __forceinline__ float finish_row(const GateParams& p, int row, int la
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams p) {
+__global__ void __launch_bounds__(kGateThreads + 32, kCtasPerSm) gate_kernel(const GateParams p) {
     __shared__ float s_m[kGateThreads / 32];
     __shared__ int s_i[kGateThreads / 32];
     __shared__ float s_S[kGateThreads / 32], s_T[kGateThreads / 32];
@@ -231,23 +258,23 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     __shared__ float s_conf[kSingleLevelMaxRows];
     __shared__ int s_arg[kSingleLevelMaxRows];
     __shared__ int s_last;
+    __shared__ __align__(8) unsigned long long s_bar[2 * kStages];
+    __shared__ volatile int s_abort;
+    __shared__ volatile int s_issued;
+    extern __shared__ __align__(128) unsigned char s_ring[];
+    const uint32_t ring0 = tc::s2u(s_ring), full0 = tc::s2u(&s_bar[0]), empty0 = tc::s2u(&s_bar[kStages]);
 
     constexpr int EPV = Loader<T>::EPV;
-    constexpr int kVStride = kGateThreads * EPV;     // columns between a thread's consecutive vectors
-    constexpr int kStep = kUnroll * kVStride;        // columns per loop iteration
     const int row = blockIdx.y, split = blockIdx.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     const T* rowp = reinterpret_cast<const T*>(p.logits) + (long long)row * p.row_stride;
     const int c0 = split * p.chunk;
     const int c_end = min(p.vocab, c0 + p.chunk);
 
-    pdl_wait();                 // the previous kernel of the stream has completed: the logits are final
-    pdl_launch_dependents();
-
     // running state: maximum, exponent base, and S, T as two packed lanes each
     float m = -INFINITY, base = base_of(-INFINITY);
     f32x2 S2 = pack2(0.f, 0.f), T2 = pack2(0.f, 0.f);
-    int mcol = -1, mspan = 0;   // where the maximum was raised: first column of the vectors to look at again, and how many
+    int mcol = -1, mspan = 0;   // where the maximum was raised: first column, and how many elements (a vector or one)
     const f32x2 kL2 = pack2(kLog2e, kLog2e);
     auto rebase_if_needed = [&](float vmax) {
         if (fmaf(vmax, kLog2e, -base) > kRebase) {   // rare
@@ -265,137 +292,136 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
         }
     };
 
-    // ---- kUnroll vectors per thread per iteration, the next kUnroll already in flight ------------------------
-    // Only the chunk's last iteration can hold vectors that are ragged or past the end; it takes the guarded path.
-    const int n_full = (c_end - c0) / kStep;
-    const int n_iter = (c_end - c0 + kStep - 1) / kStep;
-    auto fetch = [&](int it, uint4 (&raw)[kUnroll]) {
-        const int col0 = c0 + it * kStep + tid * EPV;
-        if (it < n_full) {
+    // ---- the chunk's whole vectors, staged through shared memory --------------------------------------------------
+    // Warp 8 lane 0 issues one bulk copy per stage (16 KB = four vectors per consumer thread) into a ring of kStages
+    // buffers, as far ahead as the ring allows; the bytes in flight per SM (the ring of every resident CTA) are what
+    // the pass lives on, not the consumers' registers.  Consumer thread t takes the vectors t, t + 256, t + 512, ...
+    // of the chunk in ascending order.  The ragged end of a row (a vocabulary that is no multiple of the vector
+    // length) is handled element by element below.
+    const int n_vec = (c_end - c0) / EPV;                                  // whole vectors of the chunk
+    const int n_stage = (n_vec + kStageVecs - 1) / kStageVecs;
+    if (tid == 0) {
 #pragma unroll
-            for (int v = 0; v < kUnroll; ++v) raw[v] = __ldcs(reinterpret_cast<const uint4*>(rowp + col0 + v * kVStride));   // streamed once
-        } else {
+        for (int i = 0; i < kStages; ++i) { tc::mbar_init(full0 + 8u * i, 1); tc::mbar_init(empty0 + 8u * i, kGateThreads / 32); }
+        s_abort = 0;
+        s_issued = -1;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    pdl_wait();                 // the previous kernel of the stream has completed: the logits are final
+    pdl_launch_dependents();
+    if (warp == kGateThreads / 32) {            // the producer warp
+        if (lane == 0) {
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(rowp + c0);
+            const uint64_t policy = evict_first_policy();
+            int s = 0;
+            for (; s < n_stage; ++s) {
+                const int slot = s % kStages;
+                if (s >= kStages) tc::mbar_wait(empty0 + 8u * slot, ((s / kStages) - 1) & 1, &s_abort, nullptr);
+                if (s_abort) break;
+                const uint32_t bytes = (uint32_t)min(kStageVecs, n_vec - s * kStageVecs) * 16u;
+                tc::mbar_expect_tx(full0 + 8u * slot, bytes);
+                bulk_load(ring0 + (uint32_t)slot * kStageBytes, src + (size_t)s * kStageBytes, bytes, full0 + 8u * slot, policy);
+            }
+            s_issued = s;
+        }
+        return;
+    }
+    auto consume = [&](uint4 raw, int col) {
+        Loader<T>::clamp(raw);
+        const float vmax = Loader<T>::word_max(Loader<T>::max_word(raw));
+        rebase_if_needed(vmax);
+        const bool up = vmax > m;   // strictly greater: the first vector of a tie survives
+        m = up ? vmax : m;
+        mcol = up ? col : mcol;
+        mspan = up ? EPV : mspan;
+        const f32x2 nb2 = pack2(-base, -base);
+        f32x2 x2[EPV / 2];
+        Loader<T>::widen2(raw, x2);
 #pragma unroll
-            for (int v = 0; v < kUnroll; ++v)
-                if (col0 + v * kVStride + EPV <= c_end) raw[v] = __ldcs(reinterpret_cast<const uint4*>(rowp + col0 + v * kVStride));
+        for (int i = 0; i < EPV / 2; ++i) {
+            const f32x2 d2 = fma2(x2[i], kL2, nb2);
+            float d0, d1;
+            unpack2(d2, d0, d1);
+            const f32x2 e2 = pack2(fast_exp2(d0), fast_exp2(d1));
+            S2 = add2(S2, e2);
+            T2 = fma2(e2, d2, T2);
         }
     };
-    auto consume = [&](int it, uint4 (&raw)[kUnroll]) {
-        const int col0 = c0 + it * kStep + tid * EPV;
-        if (it < n_full) {
-            unsigned int w = 0;
+    for (int s = 0; s < n_stage; ++s) {
+        const int slot = s % kStages;
+        tc::mbar_wait(full0 + 8u * slot, (s / kStages) & 1, &s_abort, nullptr);
+        if (s_abort) break;
+        const uint32_t at = ring0 + (uint32_t)slot * kStageBytes + (uint32_t)tid * 16u;
+        uint4 raw[kStageVecs / kGateThreads];
 #pragma unroll
-            for (int v = 0; v < kUnroll; ++v) {
-                Loader<T>::clamp(raw[v]);
-                const unsigned int wv = Loader<T>::max_word(raw[v]);
-                w = v == 0 ? wv : Loader<T>::max_words(w, wv);
-            }
-            const float it_max = Loader<T>::word_max(w);
-            rebase_if_needed(it_max);
-            const bool up = it_max > m;   // strictly greater: the first iteration of a tie survives
-            m = up ? it_max : m;
-            mcol = up ? col0 : mcol;
-            mspan = up ? kUnroll : mspan;
-            const f32x2 nb2 = pack2(-base, -base);
+        for (int k = 0; k < kStageVecs / kGateThreads; ++k) raw[k] = lds_v4(at + (uint32_t)k * kGateThreads * 16u);
 #pragma unroll
-            for (int v = 0; v < kUnroll; ++v) {
-                f32x2 x2[EPV / 2];
-                Loader<T>::widen2(raw[v], x2);
-#pragma unroll
-                for (int i = 0; i < EPV / 2; ++i) {
-                    const f32x2 d2 = fma2(x2[i], kL2, nb2);
-                    float d0, d1;
-                    unpack2(d2, d0, d1);
-                    const f32x2 e2 = pack2(fast_exp2(d0), fast_exp2(d1));
-                    S2 = add2(S2, e2);
-                    T2 = fma2(e2, d2, T2);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int v = 0; v < kUnroll; ++v) {
-                const int col = col0 + v * kVStride;
-                if (col >= c_end) continue;
-                float x[EPV];
-                if (col + EPV <= c_end) {
-                    Loader<T>::clamp(raw[v]);
-                    Loader<T>::widen(raw[v], x);
-                } else {   // ragged end of the row: -inf stands for "no column"
-#pragma unroll
-                    for (int i = 0; i < EPV; ++i) x[i] = (col + i < c_end) ? Loader<T>::one(rowp + col + i) : -INFINITY;
-                }
-                float vmax = x[0];
-#pragma unroll
-                for (int i = 1; i < EPV; ++i) vmax = fmaxf(vmax, x[i]);
-                rebase_if_needed(vmax);
-                const bool up = vmax > m;
-                m = up ? vmax : m;
-                mcol = up ? col : mcol;
-                mspan = up ? 1 : mspan;
-                float s0, s1, t0, t1;
-                unpack2(S2, s0, s1);
-                unpack2(T2, t0, t1);
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) {   // 2^-inf = 0, and that product is kept out of T
-                    const float d = fmaf(x[i], kLog2e, -base);
-                    const float e = fast_exp2(d);
-                    s0 += e;
-                    t0 = (x[i] == -INFINITY) ? t0 : fmaf(e, d, t0);
-                }
-                S2 = pack2(s0, s1);
-                T2 = pack2(t0, t1);
+        for (int k = 0; k < kStageVecs / kGateThreads; ++k) {
+            const int v = s * kStageVecs + k * kGateThreads + tid;
+            if (v < n_vec) consume(raw[k], c0 + v * EPV);
+        }
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(empty0 + 8u * slot);   // the stage's bytes are in registers or consumed
+    }
+    consumer_sync();
+    if (s_abort) {      // uniform: nothing raises the flag after the barrier above
+        // a wait gave up (one second): the copies already issued still target this CTA's shared memory, so the CTA
+        // stays until they have landed (bounded again) and reports through the poisoned ticket below
+        if (tid == 0) {
+            unsigned long long t0 = tc::global_timer_ns();
+            while (s_issued < 0 && tc::global_timer_ns() - t0 < tc::kWaitLimitNs) {}
+            const int issued = max(0, s_issued);
+            for (int s = max(0, issued - kStages); s < issued; ++s) {
+                t0 = tc::global_timer_ns();
+                while (!tc::mbar_try(full0 + 8u * (s % kStages), (s / kStages) & 1) && tc::global_timer_ns() - t0 < tc::kWaitLimitNs) {}
             }
         }
-    };
-    {
-        uint4 ra[kUnroll], rb[kUnroll];
-        fetch(0, ra);
-        for (int it = 0; it < n_iter; it += 2) {
-            if (it + 1 < n_iter) fetch(it + 1, rb);
-            consume(it, ra);
-            if (it + 1 < n_iter) {
-                if (it + 2 < n_iter) fetch(it + 2, ra);
-                consume(it + 1, rb);
-            }
+        consumer_sync();
+    }
+    {   // the ragged end of the chunk: fewer than EPV columns, one element per thread
+        const int col = c0 + n_vec * EPV + tid;
+        if (col < c_end) {
+            const float x = Loader<T>::one(rowp + col);
+            rebase_if_needed(x);
+            const bool up = x > m;
+            m = up ? x : m;
+            mcol = up ? col : mcol;
+            mspan = up ? 1 : mspan;
+            float s0, s1, t0, t1;
+            unpack2(S2, s0, s1);
+            unpack2(T2, t0, t1);
+            const float d = fmaf(x, kLog2e, -base);
+            const float e = fast_exp2(d);
+            S2 = pack2(s0 + e, s1);
+            T2 = pack2(fmaf(e, d, t0), t1);
         }
     }
 
     // ---- CTA-wide maximum; the threads that attained it find its first column ---------------------------
-    // every thread asks again for the vectors that raised its maximum (L2 hits, in flight during the reduction);
-    // only the threads that attained the CTA's maximum will look at them
-    uint4 again[kUnroll];
-#pragma unroll
-    for (int v = 0; v < kUnroll; ++v) {
-        again[v] = make_uint4(0u, 0u, 0u, 0u);
-        const int col = mcol + v * kVStride;
-        if (v < mspan && mcol >= 0 && col + EPV <= c_end) again[v] = __ldg(reinterpret_cast<const uint4*>(rowp + col));
-    }
+    // every thread asks again for the vector that raised its maximum (an L2 hit, in flight during the reduction); only
+    // the threads that attained the CTA's maximum will look at it
+    uint4 again = make_uint4(0u, 0u, 0u, 0u);
+    if (mspan == EPV) again = __ldg(reinterpret_cast<const uint4*>(rowp + mcol));
     float wm = m;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
     if (lane == 0) s_m[warp] = wm;
-    __syncthreads();
+    consumer_sync();
     float M = s_m[0];
 #pragma unroll
     for (int w = 1; w < kGateThreads / 32; ++w) M = fmaxf(M, s_m[w]);
     int idx = 0x7fffffff;
     if (m == M && mcol >= 0) {
+        if (mspan == EPV) {
+            float x[EPV];
+            Loader<T>::clamp(again);
+            Loader<T>::widen(again, x);
 #pragma unroll
-        for (int v = kUnroll - 1; v >= 0; --v) {   // descending: the smallest column survives
-            const int col = mcol + v * kVStride;
-            if (v >= mspan) continue;
-            if (col + EPV <= c_end) {
-                float x[EPV];
-                Loader<T>::clamp(again[v]);
-                Loader<T>::widen(again[v], x);
-#pragma unroll
-                for (int i = EPV - 1; i >= 0; --i)
-                    if (x[i] == M) idx = col + i;
-            } else {   // the chunk's ragged last vector
-#pragma unroll
-                for (int i = EPV - 1; i >= 0; --i)
-                    if (col + i < c_end && Loader<T>::one(rowp + col + i) == M) idx = col + i;
-            }
+            for (int i = EPV - 1; i >= 0; --i)   // descending: the smallest column survives
+                if (x[i] == M) idx = mcol + i;
+        } else {
+            idx = mcol;   // a single element of the ragged end
         }
     }
     // ---- sums against the CTA's base, first column of the maximum --------------------------------------
@@ -420,7 +446,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
         idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, o));
     }
     if (lane == 0) { s_S[warp] = S; s_T[warp] = Tt; s_i[warp] = idx; }
-    __syncthreads();
+    consumer_sync();
 
     // ---- publish the partial; count arrivals (tickets only count, nothing spins) --------------------
     const int seq = row / p.rows_per_seq;
@@ -431,15 +457,15 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
         for (int w = 0; w < kGateThreads / 32; ++w) { Ss += s_S[w]; Ts += s_T[w]; Midx = min(Midx, s_i[w]); }
         *reinterpret_cast<float4*>(&p.partials[(long long)row * p.splits + split]) =
             make_float4(M, Ss, Ts, __int_as_float(Midx));
-        int last;
-        if (p.single_level)
-            last = (ticket_add(&p.seq_ticket[seq], 1) == p.rows_per_seq * p.splits - 1);
-        else
-            last = (ticket_add(&p.row_ticket[row], 1) == p.splits - 1);
-        s_last = last;
+        // a CTA whose wait gave up still arrives, with the poison bit: the sequence then reports decision -1
+        const int mine = 1 + (s_abort ? kPoison : 0);
+        const int old = p.single_level ? ticket_add(&p.seq_ticket[seq], mine) : ticket_add(&p.row_ticket[row], mine);
+        const int expected = p.single_level ? p.rows_per_seq * p.splits : p.splits;
+        s_last = ((old & (kPoison - 1)) == expected - 1 ? 1 : 0) | (old + mine >= kPoison ? 2 : 0);
     }
-    __syncthreads();   // orders the ticket's acquire before the other threads' reads of the partials
-    if (!s_last) return;
+    consumer_sync();   // orders the ticket's acquire before the other threads' reads of the partials
+    if (!(s_last & 1)) return;
+    const bool poisoned = (s_last & 2) != 0;
 
     if (p.single_level) {
         // ---- last CTA of the sequence: finish every row, then the masked maximum and the decision ----
@@ -488,7 +514,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                 }
             }
         }
-        __syncthreads();
+        consumer_sync();
         if (warp == 0 && p.masked) {
             // ---- confidence-based parallel decoding (Section 2.1 of the paper; threshold 0.9 in its experiments):
             // every masked row above the threshold is decoded; if none is, the masked row of highest confidence
@@ -539,7 +565,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                 if (p.ent_sum_out) p.ent_sum_out[seq] = Hsum;
                 if (p.max_conf_out) p.max_conf_out[seq] = Cmax;
                 p.max_entropy_out[seq] = E;
-                p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
+                p.decision_out[seq] = poisoned ? -1 : (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
                 p.seq_ticket[seq] = 0;   // ready for the next call
             }
         } else if (warp == 0) {
@@ -559,7 +585,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
                 if (p.ent_sum_out) p.ent_sum_out[seq] = Hsum;
                 if (p.max_conf_out) p.max_conf_out[seq] = Cmax;
                 p.max_entropy_out[seq] = E;
-                p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
+                p.decision_out[seq] = poisoned ? -1 : (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
                 p.seq_ticket[seq] = 0;   // ready for the next call
             }
         }
@@ -572,10 +598,12 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     int seq_last = 0;
     if (lane == 0) {
         p.row_ticket[row] = 0;
-        seq_last = (ticket_add(&p.seq_ticket[seq], 1) == p.rows_per_seq - 1);
+        const int mine = 1 + (poisoned ? kPoison : 0);
+        const int old = ticket_add(&p.seq_ticket[seq], mine);
+        seq_last = ((old & (kPoison - 1)) == p.rows_per_seq - 1 ? 1 : 0) | (old + mine >= kPoison ? 2 : 0);
     }
     seq_last = __shfl_sync(0xffffffffu, seq_last, 0);
-    if (!seq_last) return;
+    if (!(seq_last & 1)) return;
     float E = -INFINITY;
     for (int r = lane; r < p.rows_per_seq; r += 32) {
         const int rr = seq * p.rows_per_seq + r;
@@ -585,7 +613,7 @@ __global__ void __launch_bounds__(kGateThreads, 4) gate_kernel(const GateParams 
     for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
     if (lane == 0) {
         p.max_entropy_out[seq] = E;
-        p.decision_out[seq] = (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
+        p.decision_out[seq] = (seq_last & 2) ? -1 : (E > p.tau) ? EC_RECOMPUTE : EC_SKIP;
         p.seq_ticket[seq] = 0;
     }
 }
@@ -609,7 +637,7 @@ GateWs carve(int n_rows) {
 // of 2048-column slabs, at most kMaxSplits partials per row
 void plan_chunks(int n_rows, int vocab, int* splits, int* chunk, int max_splits = kMaxSplits) {
     const int slab = kGateThreads * kVec;
-    const long long slots = 4LL * sm_count();
+    const long long slots = (long long)kCtasPerSm * sm_count();
     long long want = slots / n_rows;
     if (want < 1) want = 1;
     if (want > max_splits) want = max_splits;
@@ -625,8 +653,11 @@ template <typename T>
 cudaError_t launch_t(const GateParams& p, cudaStream_t stream) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(p.splits, p.n_rows, 1);
-    cfg.blockDim = dim3(kGateThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
+    cfg.blockDim = dim3(kGateThreads + 32, 1, 1);    // the consumer warps and the producer warp
+    cfg.dynamicSmemBytes = kStages * kStageBytes;
+    static PerDeviceOnce once;
+    const cudaError_t e = ensure_dynamic_smem(once, gate_kernel<T>, kStages * kStageBytes);
+    if (e != cudaSuccess) return e;
     cfg.stream = stream;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // launch latency may overlap the previous kernel's tail
