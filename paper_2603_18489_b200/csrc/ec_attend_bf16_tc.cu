@@ -26,6 +26,7 @@
 // caller's dev_status word, raises a CTA-wide abort flag that makes all later
 // waits fall through, and the CTA still frees its TMEM and exits.
 #include "ec_common.cuh"
+#include "ec_tc_ptx.cuh"
 
 #include <cuda.h>
 
@@ -42,7 +43,6 @@ constexpr uint32_t OFF_V = OFF_K + 2 * TILE;     // 2 stages
 constexpr uint32_t OFF_P = OFF_V + 2 * TILE;     // 2 buffers
 constexpr uint32_t OFF_BAR = OFF_P + 2 * TILE;   // 224 KiB
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256 + 1024;  // + barrier block + alignment slack
-constexpr uint32_t kSpinLimit = 1u << 22;        // polls per wait before giving up
 
 constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;
 
@@ -50,41 +50,19 @@ constexpr uint32_t TM_S0 = 0, TM_S1 = 128, TM_O = 256, TM_COLS = 512;
 enum { B_KFULL = 0, B_KEMPTY = 2, B_VFULL = 4, B_VEMPTY = 6, B_SFULL = 8, B_PFULL = 10, B_PVDONE = 12, B_COUNT = 14 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
-__device__ __forceinline__ uint32_t s2u(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// bounded wait; on failure raises the CTA's abort flag (and every later wait returns at once)
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try(bar, parity)) return;
-        if ((i & 63) == 63 && *abort_flag) return;
-    }
-    *abort_flag = 1;
-    if (dev_status) atomicExch(dev_status, (int)EC_ERR_TIMEOUT);
-}
+// mbarriers (bounded waits), shared-memory addresses and the async-proxy fence are the shared wrappers
+using tc::s2u;
+using tc::mbar_init;
+using tc::mbar_arrive;
+using tc::mbar_expect_tx;
+using tc::mbar_try;
+using tc::mbar_wait;
+using tc::fence_async_smem;
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -424,22 +402,8 @@ __global__ void __launch_bounds__(128) attend_tc_combine_kernel(const TcParams p
 }
 
 // ---- host side ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
+using tc::EncodeTiledFn;
+using tc::encode_fn;
 
 // cache [B*Hkv, L, 128] bf16 -> 3-D map {d, key, head}; box {64, 128, 1}; 128-byte swizzle; keys beyond L read as zero
 bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {

@@ -9,7 +9,7 @@
 //               [64 columns], 128-byte swizzle) through a ring of five 32 KB slots (K0 V0 K1 V1 ...), and the
 //               two Q tiles of the unit, one box each.  (Grouped-query shapes are launched with one unit per
 //               QUERY head, so a row tile is always 128 active rows of one head; the query heads of a kv head
-//               stream the same K/V, which L2 serves.  The thread-staged Q path below remains for packed tiles.)
+//               stream the same K/V, which L2 serves.)
 //   warp 1      tcgen05.mma issuer (one thread): S_t = Q_t K^T (both operands K-major in shared memory) into
 //               the TMEM columns of row tile t, and O_t += P_t V with P_t read from TENSOR MEMORY (it
 //               overwrites the first 64 columns of S_t as packed bf16) and V MN-major from shared memory.
@@ -43,7 +43,6 @@ using namespace tc;
 constexpr int BM = 128, BN = 128, HD = 128;
 constexpr int kSoftThreads = 512;          // four softmax warpgroups: (row tile) x (64-column half)
 constexpr int kThreads = 64 + kSoftThreads + 32;   // + one warp that copies fresh K/V into the cache (recompute steps)
-constexpr int kPolyOf5 = 0;                // pairs out of every five whose exponentials go to the FMA pipe
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr int kSlots = 5;
@@ -59,28 +58,6 @@ constexpr uint32_t TM_S = 0, TM_O = 256;   // + 128 * tile
 enum { B_FULL = 0, B_EMPTY = kSlots, B_SFULL = 2 * kSlots, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_COUNT = B_QFULL + 1 };
 
-// 2^x for a pair of values on the FMA pipe (the MUFU pipe is the softmax's bottleneck, so a share of the
-// exponentials is computed here instead): x = n + f with n = round(x), |f| <= 1/2, 2^f by a cubic fitted for a
-// maximum relative error of 7.5e-5 (far below the bf16 rounding of P), and n added to the exponent field.
-// Inputs below -126 give (flushed) zero.
-__device__ __forceinline__ void exp2_poly2(f32x2 d2, float& e0, float& e1) {
-    float x0, x1;
-    upk(d2, x0, x1);
-    const f32x2 x2 = pk(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-    const f32x2 magic2 = pk(12582912.f, 12582912.f);   // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
-    const f32x2 t2 = add2(x2, magic2);
-    const f32x2 n2 = add2(t2, pk(-12582912.f, -12582912.f));
-    const f32x2 f2 = fma2(n2, pk(-1.f, -1.f), x2);
-    f32x2 p2 = fma2(f2, pk(0.05517146f, 0.05517146f), pk(0.24261086f, 0.24261086f));
-    p2 = fma2(p2, f2, pk(0.69326097f, 0.69326097f));
-    p2 = fma2(p2, f2, pk(0.9999281f, 0.9999281f));
-    float p0, p1, t0, t1;
-    upk(p2, p0, p1);
-    upk(t2, t0, t1);
-    e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-    e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-}
-
 struct DenseParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
@@ -92,7 +69,6 @@ struct DenseParams {
     uint4* v_dst;
     int32_t* dev_status;
     int n_active, ctx_len, n_q_heads, n_kv_heads, group, rows_total;
-    int q_tma;   // 1: one query head per kv head, the producer fetches the Q tiles with one TMA box each
     // Grouped-query shapes run with one unit per QUERY head (the kernel then sees n_kv_heads = n_q_heads = H_q and
     // group = 1, so its row tiles are 128 active rows of one head and come by TMA); the K/V of unit head h are
     // those of the real kv head h / kv_div, of which there are n_kv_real.  kv_div = 1 otherwise.
@@ -127,7 +103,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         prefetch_map(&map_k);
         prefetch_map(&map_v);
         for (int i = 0; i < B_COUNT; ++i)
-            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 256u : (i == B_QFULL && !p.q_tma ? (uint32_t)kSoftThreads : 1u));
+            mbar_init(bar(i), (i >= B_PFULL && i < B_PFULL + 2) ? 256u : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -147,12 +123,11 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // ================================ TMA producer ======================================
         if (lane == 0) {
             const int hk_kv = hk / p.kv_div;
-            if (p.q_tma) {   // Q first: [half][row][64 columns] per row tile; rows past n_active read as zero
-                prefetch_map(&map_q);
-                mbar_expect_tx(bar(B_QFULL), (uint32_t)n_tiles_q * TILE);
-                for (int t = 0; t < n_tiles_q; ++t)
-                    tma_load_5d(base + OFF_Q + t * TILE, &map_q, 0, r_pair + t * BM, hk, 0, b, bar(B_QFULL));
-            }
+            // Q first: [half][row][64 columns] per row tile; rows past n_active read as zero
+            prefetch_map(&map_q);
+            mbar_expect_tx(bar(B_QFULL), (uint32_t)n_tiles_q * TILE);
+            for (int t = 0; t < n_tiles_q; ++t)
+                tma_load_5d(base + OFF_Q + t * TILE, &map_q, 0, r_pair + t * BM, hk, 0, b, bar(B_QFULL));
             for (int n = 0; n < 2 * T; ++n) {   // ring index: K_j = 2j, V_j = 2j + 1
                 const int slot = n % kSlots, u = n / kSlots;
                 if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
@@ -199,27 +174,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
         }
     } else if (warp < 2 + kSoftThreads / 32) {
-        // ============== Q staging (GQA shapes only), then softmax (warps 2..17) ===============
-        const int stid = tid - 64;
-        if (!p.q_tma) {
-            // Q rows of this kv head -> two swizzled K-major tiles (rows beyond rows_total are zero)
-            for (int c = stid; c < 2 * BM * (HD / 8); c += kSoftThreads) {
-                const int row = c >> 4, ch = c & 15;   // row in [0, 256)
-                const int r = r_pair + row;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (r < p.rows_total) {
-                    const int i = r / p.group, j = r % p.group;
-                    v = __ldg(reinterpret_cast<const uint4*>(
-                        p.q + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + j) * HD + ch * 8));
-                }
-                const int t = row >> 7, rt = row & 127;
-                const uint32_t off = OFF_Q + t * TILE + (ch >> 3) * SUB + (rt >> 3) * 1024 + (rt & 7) * 128 + (((ch & 7) ^ (rt & 7)) << 4);
-                *reinterpret_cast<uint4*>(gbase + off) = v;
-            }
-            fence_async_smem();   // generic-proxy writes of Q -> visible to the tensor core (async proxy)
-            mbar_arrive(bar(B_QFULL));
-        }
-
+        // ================================ softmax (warps 2..17) ================================
         // A row of a tile is shared by two threads, one per 64-column half, in warps that own the same TMEM
         // lanes: softmax warp ws = warp - 2 -> row tile ws / 8, column half (ws / 4) % 2, lanes 32 * (warp % 4).
         const int ws = warp - 2;
@@ -271,15 +226,9 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const f32x2 d2 = fma2(pk(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), sl2_2, mneg2);
-                    float e0, e1;
-                    if (kPolyOf5 > 0 && c % 5 < kPolyOf5) {   // this share of the pairs on the FMA pipe, the rest on the MUFU pipe
-                        exp2_poly2(d2, e0, e1);
-                    } else {
-                        float d0, d1;
-                        upk(d2, d0, d1);
-                        e0 = fast_exp2(d0);
-                        e1 = fast_exp2(d1);
-                    }
+                    float d0, d1;
+                    upk(d2, d0, d1);
+                    const float e0 = fast_exp2(d0), e1 = fast_exp2(d1);
                     sum2[c & 1] = add2(sum2[c & 1], pk(e0, e1));
                     pw[c] = pack_bf16x2(e0, e1);
                 }
@@ -442,9 +391,8 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     p.kv_div = a.d.n_q_heads / a.d.n_kv_heads;
     p.n_kv_real = a.d.n_kv_heads;
     p.scale_log2 = a.scale * kLog2e;
-    p.q_tma = 1;
-    CUtensorMap map_q = map_k;   // unused unless q_tma
-    if (p.q_tma) {
+    CUtensorMap map_q;
+    {
         EncodeTiledFn fn = encode_fn();
         if (!fn) return cudaErrorInvalidValue;
         const cuuint64_t dims[5] = {64, (cuuint64_t)a.n_active, (cuuint64_t)a.d.n_q_heads, 2, (cuuint64_t)a.d.batch};

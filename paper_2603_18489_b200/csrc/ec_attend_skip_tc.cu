@@ -43,6 +43,7 @@
 // caller's dev_status word and a CTA-wide abort flag that makes all later waits fall
 // through; the CTA still frees its TMEM and exits.
 #include "ec_common.cuh"
+#include "ec_tc_ptx.cuh"
 
 #include <cuda.h>
 
@@ -57,7 +58,6 @@ constexpr uint32_t KV_TILE = 2 * KV_SUB;   // [64 keys x 128 bf16]
 constexpr uint32_t STAGE = 2 * KV_TILE;    // K tile + V tile: 32 KB
 constexpr int kMaxStages = 6;
 constexpr int kRec = HD + 4;               // floats per exchanged row: O[128], m, l, pad (16-byte multiple)
-constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kMaxRows = 2 * BM;
 constexpr int kMaxCluster = 8;
 
@@ -76,34 +76,14 @@ enum {
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
-__device__ __forceinline__ uint32_t s2u(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try(bar, parity)) return;
-        if ((i & 63) == 63 && *abort_flag) return;
-    }
-    *abort_flag = 1;
-    if (dev_status) atomicExch(dev_status, (int)EC_ERR_TIMEOUT);
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// mbarriers (bounded waits), shared-memory addresses and the async-proxy fence are the shared wrappers
+using tc::s2u;
+using tc::mbar_init;
+using tc::mbar_arrive;
+using tc::mbar_expect_tx;
+using tc::mbar_try;
+using tc::mbar_wait;
+using tc::fence_async_smem;
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -665,22 +645,8 @@ attend_skip_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 }
 
 // ---- host side ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
+using tc::EncodeTiledFn;
+using tc::encode_fn;
 
 // cache [B*Hkv, L, 128] bf16 seen as 4-D {64 columns, key, half, head}: one box {64, 64, 2, 1} lands as
 // [half][key][64 columns], i.e. the two 128-byte-swizzled halves of a [64 keys x 128] tile back to back; keys
