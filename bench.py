@@ -49,33 +49,40 @@ PER_WORKLOAD = ("c2_llada_l768", "c3_dream_l768", "c4_llada_l2048", "c5_llada_l4
 K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dream_l4096")   # also timed at the paper's k = 64
 
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/.  A figure is reported only while the kernel's source file still has the hash it had when the
+# DRAM traffic per launch (reads + writes: dram__bytes.sum.per_second x gpu__time_duration.sum) from the ncu captures
+# summarised under profiles/.  A figure is reported only while the kernel's source file still has the hash it had when the
 # counters were taken; after any change to the kernel it reads null until the capture is redone.
 NCU_TRAFFIC = {
-    "attend_skip": {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-                    "sha256": "e9aff5110c7667b8ad12c758605c719f594430da1eacc5bb078ee95d7f223974",
-                    "bytes_per_launch": {"c2_llada_l768": 12968960, "c5_llada_l4096": 68200704}},
-    "attend_dense": {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
-                     "sha256": "54ec597014094429ac7064859b7b2ca2a2537ad8867d42cc57f9e8822b2caf58",
-                     "bytes_per_launch": {"c2_llada_l768": 18928896, "c4_llada_l2048": 60230144, "c5_llada_l4096": 161412864}},
-    "entropy_gate": {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
-                     "sha256": "7d578bb920ed3bc65f911bb747e22b6bb333a6dfcdf62f16dc30489f58ce07e4",
-                     "bytes_per_launch": {"c2_llada_l768": 8160768, "c5_llada_l4096_b8": 65172992}},
+    "attend_skip": [
+        {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
+         "sha256": "c0f749f309b62c7b5fc80e0e0a119662d86d17899842bae0e7c8816b83bc9011",
+         "bytes_per_launch": {"c2_llada_l768": 13520000, "c5_llada_l4096": 68080000}},
+        {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
+         "sha256": "0675aade2351435060878966d4be0572ffac430f9a3166b6c13a657a9dbbd731",
+         "bytes_per_launch": {"c5_llada_l4096_b8": 552370000}}],
+    "attend_dense": [
+        {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
+         "sha256": "9633a97b1fa145586220abd4f95827e8d6e35f1c6512fcb5089beec8b73980a4",
+         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62860000}}],
+    "entropy_gate": [
+        {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
+         "sha256": "9aff17035d14500e5378489b0f9cb64e1b4f42fbe658d39056e2c7edeb701d42",
+         "bytes_per_launch": {"c5_llada_l4096": 8140000, "c5_llada_l4096_b8": 65130000}}],
 }
 
 
 def _ncu_traffic(kernel: str, workload: str):
     import hashlib
 
-    e = NCU_TRAFFIC[kernel]
-    try:
-        h = hashlib.sha256(open(os.path.join(ROOT, e["source"]), "rb").read()).hexdigest()
-    except OSError:
-        return None
-    if h != e["sha256"]:
-        return None
-    return e["bytes_per_launch"].get(workload)
+    for e in NCU_TRAFFIC[kernel]:
+        if workload not in e["bytes_per_launch"]:
+            continue
+        try:
+            h = hashlib.sha256(open(os.path.join(ROOT, e["source"]), "rb").read()).hexdigest()
+        except OSError:
+            return None
+        return e["bytes_per_launch"][workload] if h == e["sha256"] else None
+    return None
 
 
 def _peaks() -> dict:
