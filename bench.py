@@ -55,7 +55,7 @@ K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dr
 NCU_TRAFFIC = {
     "attend_skip": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-         "sha256": "c0f749f309b62c7b5fc80e0e0a119662d86d17899842bae0e7c8816b83bc9011",
+         "sha256": "9bd232c483760aa0025407450b8a1a8910575385e76598e26f0634f11907660a",
          "bytes_per_launch": {"c2_llada_l768": 13520000, "c5_llada_l4096": 68080000}},
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
          "sha256": "0675aade2351435060878966d4be0572ffac430f9a3166b6c13a657a9dbbd731",
@@ -63,7 +63,7 @@ NCU_TRAFFIC = {
     "attend_dense": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
          "sha256": "9633a97b1fa145586220abd4f95827e8d6e35f1c6512fcb5089beec8b73980a4",
-         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62860000}}],
+         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62860000, "c5_llada_l4096": 163660000}}],
     "entropy_gate": [
         {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
          "sha256": "9aff17035d14500e5378489b0f9cb64e1b4f42fbe658d39056e2c7edeb701d42",

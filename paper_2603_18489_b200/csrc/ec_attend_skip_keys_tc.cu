@@ -8,16 +8,15 @@
 // axis (N = 48, 64 or 96 slots):
 //     S^T[128 keys x N]  = K_tile[128 keys x 128] . Q[N x 128]^T          (A = K tile, B = Q, both K-major)
 //     O^T[128 d    x N] += V_tile^T[128 d x 128 keys] . P^T[128 keys x N]  (A = V tile MN-major, B = P^T MN-major)
-//     L^T[128      x N] += 1[128 x 128 keys]          . P^T[128 keys x N]  (A = a block of ones in tensor memory)
 // so a softmax thread owns one KEY (TMEM lane) and its scores against the query slots: all 128 lanes work, one
-// exponential per (key, query), no padding rows, a pipeline step covers 128 keys.  The row sums come out of the
-// tensor core as well (every lane of L^T holds sum_keys P), so the softmax threads carry no running sums and
-// nothing has to be reduced across threads at the end.  With N = 96 (the paper's default budget k = 64 gives 96
-// active rows) two softmax warpgroups share the columns of a key.
+// exponential per (key, query), no padding rows, a pipeline step covers 128 keys.  The row sums sum_keys P are
+// taken by two auxiliary warps that read P^T back from shared memory (where the softmax threads put it for the
+// second product), so the softmax threads carry no running sums.  With N = 96 (the paper's default budget k = 64
+// gives 96 active rows) two softmax warpgroups share the columns of a key.
 //   softmax  the reference maxima m[q] (log2 units) are shared by all keys of the CTA and live in shared memory.
 //            The common path computes p = 2^(s*scale*log2e - m[q]) with no reduction at all; a barrier-wide OR
 //            tells whether any score exceeds its reference by more than 2^8 (always true on the first tile):
-//            only then the column maxima are reduced, m is raised, and O^T and L^T are rescaled;
+//            only then the column maxima are reduced, m is raised, and O^T and the row sums are rescaled;
 //   grid     (C, B*H_kv*n_sub) as clusters of C <= 8 CTAs (any count, not only powers of two) that split one
 //            head's 128-key tiles, chosen so that the most-loaded SM streams the fewest tiles; CTAs that hold a
 //            single tile are small enough for two per SM.  With grouped-query attention the query heads of a kv
@@ -30,13 +29,16 @@
 //            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) before its cache
 //            tiles, while every CTA masks the stale cached keys of the refreshed positions (a bit per key, built from
 //            the index list).  The attention therefore never waits for the cache update: the auxiliary warps of that
-//            CTA copy the fresh rows into the cache in global memory for later steps, ordered against nothing.  (Keys
+//            CTA send the fresh rows from the landed tile to the cache in global memory, one TMA row store per row
+//            and half, for later steps, ordered against nothing.  (Keys
 //            in a different order, the same sum.)  When a CTA holds a single cache tile the extra tiles get a CTA of
 //            their own, so that nobody streams two tiles through one stage;
 //   merge    CTA c of the cluster owns the output columns d in [c*DL, (c+1)*DL): once every CTA of the cluster is
-//            past its main loop (first cluster barrier) each softmax thread stores its O^T row (one output column,
-//            all queries) straight into the owner's shared memory, plus m and l; after the second cluster barrier
-//            the owner combines the C partials, normalises and writes out[b, i, h, d].
+//            past its last product (first cluster barrier, arrive early / wait late) each softmax thread puts its
+//            O^T row (one output column, all queries) into a local staging chunk per owner, next to m and l; one
+//            bulk copy per owner moves the chunk into the owner's shared memory and completes on the owner's
+//            mbarrier; the owner combines the C partials, normalises and writes out[b, i, h, d]; a second cluster
+//            barrier keeps every CTA's shared memory alive until its peers have read it.
 // warp 0: TMA producer; warp 1: stale-key masks, then tcgen05.mma issue; next 4 (or 8) warps: softmax; last two
 // warps: cache update and row sums.  Launched with programmatic stream serialisation; global memory is touched only after
 // griddepcontrol.wait.  Every mbarrier wait is bounded (EC_ERR_TIMEOUT in dev_status, CTA-wide abort flag: an
