@@ -260,7 +260,12 @@ ec_status ec_select_recent(int32_t *history, int32_t ctx_len, int32_t batch, ec_
  *   4. active_idx[b, :] = the first `window` positions with masked[b, pos] != 0, ascending (fewer when fewer
  *      remain), then the positions of R ascending (a decoded position is never masked, so the two are disjoint),
  *      then -1 up to n_cap; state[b].n_active = their count (beyond n_cap the list is cut, as in ec_select_recent).
- * masked: uint8 [batch, ctx_len], in/out; the other arguments as for ec_select_recent. */
+ * masked: uint8 [batch, ctx_len], in/out; the other arguments as for ec_select_recent.
+ * Between two calls the caller changes neither `masked` nor active_idx: the size of the current window is recomputed
+ * as min(window, number of masked positions of the sequence), and its rows are read back from active_idx[b, 0 : that
+ * size].  Before the first call the caller writes exactly that many entries, the first masked positions in ascending
+ * order.  A sequence whose current window holds an entry that is out of range or no longer masked is left untouched
+ * (history, masked, state, list) except for state[b].n_active = -1. */
 ec_status ec_select_recent_sliding(int32_t *history, int32_t ctx_len, int32_t batch, ec_step_state *state,
                                    uint8_t *masked, const uint8_t *decoded_flags, int32_t window,
                                    const int32_t *decision, int32_t k, int32_t *active_idx, int32_t n_cap,

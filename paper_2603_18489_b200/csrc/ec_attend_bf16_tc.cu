@@ -329,7 +329,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                 float o[32];
                 tc_ld32(tmem + lane_addr + TM_O + c * 32, o);
                 tc_wait_ld();
-                if (valid) {
+                if (valid && !*abort_flag) {   // a CTA whose wait gave up stores nothing
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         uint4 w;

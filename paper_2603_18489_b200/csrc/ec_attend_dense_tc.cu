@@ -274,7 +274,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 uint32_t o[32];
                 ld32(tm_o + h * 64 + c * 32, o);
                 wait_ld();
-                if (valid) {
+                if (valid && !*abort_flag) {   // a CTA whose wait gave up stores nothing
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         uint4 w;

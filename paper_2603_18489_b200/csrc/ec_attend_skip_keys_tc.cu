@@ -22,8 +22,9 @@
 //            single tile are small enough for two per SM.  With grouped-query attention the query heads of a kv
 //            head are packed into the N axis; when they exceed the slots the heads (and, beyond 96 active rows,
 //            the rows) are spread over n_sub CTA columns that stream the same K/V (L2 serves the repeats);
-//   K/V      the producer warp issues its TMA loads at once, in key order, through a ring of NS stages of 64 KB:
-//            they depend on nothing;
+//   K/V      the producer warp issues its TMA loads in key order through a ring of NS stages of 64 KB; they depend on
+//            nothing, and the first fill of the ring is spaced in time (one stage of every CTA per interval) so
+//            that the memory system always has requests queued while the first tiles are consumed;
 //   refresh  the active rows' fresh K/V reach the attention straight from k_new / v_new, not through the cache: one
 //            CTA of every cluster (the last) attends to them as one or two EXTRA key tiles, fetched by TMA from the
 //            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) before its cache
@@ -125,6 +126,10 @@ struct KeysParams {
     uint32_t off_p, off_stage, off_list, off_bar;   // shared-memory carve (bytes from the 1024-aligned base); Q is at 0;
                                                     // off_list: the stale-key bits, 16 bytes per refreshed cache tile
     float scale_log2;
+    // Nanoseconds the memory system needs for one stage of every CTA that streams its own K/V: the producer spaces
+    // the first fill of its ring by this much per stage, so that the stages of the launch arrive one wave after the
+    // other instead of all together (0: no spacing).
+    uint32_t stagger_ns;
 };
 
 // words after the barrier block
@@ -234,8 +239,17 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
                 tma_load_5d(base, &map_q, 0, i0, hq0, 0, b, bar(B_QFULL));   // rows past the chunk land in unused slots
             }
+            const unsigned long long t_fill = global_timer_ns();
             for (int j = 0; j < T; ++j) {
                 const int s = j % NS, u = j / NS;
+                if (u == 0 && j > XT && p.stagger_ns) {
+                    // First fill of the ring: cache stage c of every CTA is asked for c * stagger_ns after the first, so
+                    // the first tiles of all CTAs land before anybody's second, and requests stay queued while they
+                    // are consumed.  (Asked for all at once, the stages of the whole launch arrive together after
+                    // the time of all of them, and the memory system then idles until the first stage is free again.)
+                    const unsigned long long due = t_fill + (unsigned long long)(j - XT) * p.stagger_ns;
+                    while (global_timer_ns() < due) __nanosleep(64);
+                }
                 if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
                 if (u > 0 && j - NS < XT && sub == 0)   // the stage held a fresh tile: the cache update has read it
                     mbar_wait(bar(B_FRESHOUT + (j - NS)), 0, abort_flag, p.dev_status);   // (one single-phase barrier per fresh tile)
@@ -879,6 +893,29 @@ bool make_fresh_map(CUtensorMap* map, const void* fresh, int batch, int n_active
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bytes per nanosecond assumed for a streaming read when spacing the first ring fill: 0.7 of the nominal rate of the
+// device (clock x bus width, double data rate; a spacing between 1.0 and 1.3 times the measured copy rate's stage
+// time timed best), cached per device
+double stream_bytes_per_ns() {
+    static std::atomic<uint64_t> cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 5700.0;
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    if (slot) {
+        const uint64_t v = cached[dev].load(std::memory_order_relaxed);
+        if (v) return (double)v;
+    }
+    int khz = 0, bits = 0;
+    if (cudaDeviceGetAttribute(&khz, cudaDevAttrMemoryClockRate, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&bits, cudaDevAttrGlobalMemoryBusWidth, dev) != cudaSuccess || khz <= 0 || bits <= 0) {
+        (void)cudaGetLastError();
+        return 5700.0;
+    }
+    const double rate = 0.7 * 2.0 * (double)khz * 1e3 * (bits / 8.0) * 1e-9;
+    if (slot) cached[dev].store((uint64_t)rate, std::memory_order_relaxed);
+    return rate;
+}
+
 template <int N>
 cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv,
                      const CUtensorMap& mq, const CUtensorMap& mkn, const CUtensorMap& mvn, const CUtensorMap& mk1,
@@ -966,6 +1003,12 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.off_list = pl.off_list;
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
+    p.stagger_ns = 0;
+    if (pl.tiles_per_split > 1) {
+        const double streams = (double)pl.n_splits * bh;   // CTAs with K/V of their own (columns of one head share it through L2)
+        const double ns = streams * STAGE / stream_bytes_per_ns();
+        p.stagger_ns = (uint32_t)(ns < 3000.0 ? ns : 3000.0);
+    }
     const int cols = bh * pl.n_sub;
     return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)
            : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)

@@ -537,7 +537,7 @@ attend_skip_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                     float o[32];
                     tc_ld32(tm_t + 128 + c * 32, o);
                     tc_wait_ld();
-                    if (valid) {
+                    if (valid && !*abort_flag) {   // a CTA whose wait gave up stores nothing
 #pragma unroll
                         for (int v4 = 0; v4 < 4; ++v4) {
                             uint4 w;
@@ -627,7 +627,7 @@ attend_skip_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
                 uint2 w2;
                 w2.x = pack2(acc.x * inv, acc.y * inv);
                 w2.y = pack2(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(dst + lane * 4) = w2;
+                if (!*abort_flag) *reinterpret_cast<uint2*>(dst + lane * 4) = w2;   // nothing from a CTA whose wait gave up
             }
         }
         // no CTA leaves while a peer may still copy out of or into its shared memory

@@ -7,7 +7,8 @@
 //   min over K   history values are step indices <= t, so the k-th largest value is found by bisection on the
 //                value: the largest v in [vmin, t] with |{i : H_i >= v}| >= k; each probe is one block-wide count.
 //                If fewer than k positions were ever decoded the minimum is "-infinity" and only t - dt limits R.
-// The kernel has no waits; an out-of-range window leaves the sequence untouched and reports n_active = -1.
+// The kernel has no waits; an out-of-range window (block mode) or a window list that does not consist of masked
+// positions (sliding mode) leaves the sequence untouched and reports n_active = -1.
 #include "ec_common.cuh"
 
 namespace ec {
@@ -67,6 +68,20 @@ __global__ void __launch_bounds__(kSelThreads) select_recent_kernel(const Select
         c = block_sum(c, scratch);
         n_cur = c < p.block ? c : p.block;
         __syncthreads();
+        // the window rows must be the list the previous call (or, before the first call, the caller) wrote: in range
+        // and still masked.  Anything else would credit the decoded flags to the wrong positions, so the sequence is
+        // left untouched and reports n_active = -1, as an out-of-range window does in block mode.
+        int bad = 0;
+        for (int r = tid; r < n_cur; r += kSelThreads) {
+            const int pos = idx[r];
+            bad += (pos < 0 || pos >= p.ctx_len || M[pos] == 0) ? 1 : 0;
+        }
+        bad = block_sum(bad, scratch);
+        __syncthreads();
+        if (bad) {   // uniform over the CTA
+            if (tid == 0) p.state[b].n_active = -1;
+            return;
+        }
     }
     // ---- Eq. 2: the positions decoded in this step get the step's index -----------------------------
     // block mode: window row r is position w0 + r; sliding mode: it is entry r of the row list of the previous call

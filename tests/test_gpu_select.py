@@ -150,3 +150,40 @@ def test_sliding_window_traces_match_the_oracle(B, L, prompt, window, k):
 def test_sliding_window_runs_out_of_masked_positions():
     """40 positions to generate, window 16: after a few steps fewer than 16 remain and the window shrinks to what is left."""
     _sliding_trace(1, 140, 100, 16, 4, n_steps=40, seed=77, n_cap=16 + 64)
+
+
+def test_sliding_window_list_that_is_not_masked_positions_is_rejected_per_sequence():
+    """Sequence 0 is seeded with its proper first window, sequence 1 with a list that names an already decoded
+    position, sequence 2 with an out-of-range entry: the first proceeds as the oracle says, the other two are left
+    untouched and report n_active = -1 (the rule an out-of-range window follows in block mode)."""
+    import paper_2603_18489_b200 as ec
+
+    B, L, prompt, window, k, n_cap = 3, 256, 100, 16, 2, 64
+    dev = torch.device("cuda")
+    hist, state = ec.new_history(B, L), ec.new_step_state(B, 1)
+    masked_np = np.ones((B, L), np.uint8)
+    masked_np[:, :prompt] = 0
+    masked = torch.from_numpy(masked_np.copy()).to(dev)
+    first = oracle.sliding_window_rows(masked_np[0], window).astype(np.int32)
+    lists = np.full((B, n_cap), -1, np.int32)
+    lists[0, :window] = first
+    lists[1, :window] = first
+    lists[1, 3] = 7                      # a prompt position: not masked
+    lists[2, :window] = first
+    lists[2, 5] = L + 4                  # out of range
+    idx = torch.from_numpy(lists.copy()).to(dev)
+    flags = np.zeros((B, window), np.uint8)
+    flags[:, [1, 3, 5]] = 1
+    dec = np.zeros(B, np.int32)
+    ec.ec_select_recent_sliding(hist, state, masked, torch.from_numpy(flags.reshape(-1)).to(dev), window,
+                                torch.from_numpy(dec).to(dev), k, idx)
+    torch.cuda.synchronize()
+    g_hist, g_state, g_idx, g_m = hist.cpu().numpy(), state.cpu().numpy(), idx.cpu().numpy(), masked.cpu().numpy()
+    H, M = np.full(L, -np.inf), masked_np[0].copy()
+    new_rows, skip, dt, t = oracle.sliding_step_bookkeeping(H, M, 1, 0, first.astype(np.int64), flags[0], 0, k, window)
+    assert g_state[0].tolist() == [t, dt, int(skip), new_rows.size]
+    assert g_idx[0, :new_rows.size].tolist() == new_rows.tolist() and np.array_equal(g_m[0], M)
+    for b in (1, 2):
+        assert g_state[b].tolist() == [1, 0, 0, -1]
+        assert (g_hist[b] == NEVER).all() and np.array_equal(g_m[b], masked_np[b])
+        assert np.array_equal(g_idx[b], lists[b])
