@@ -55,15 +55,15 @@ K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dr
 NCU_TRAFFIC = {
     "attend_skip": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-         "sha256": "9bd232c483760aa0025407450b8a1a8910575385e76598e26f0634f11907660a",
-         "bytes_per_launch": {"c2_llada_l768": 13520000, "c5_llada_l4096": 68080000}},
+         "sha256": "4e4c7fc5a90767439edacee25758e74549d67d3e91ef33574a4fd8ca09109af3",
+         "bytes_per_launch": {"c2_llada_l768": 13510000, "c5_llada_l4096": 68160000}},
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
-         "sha256": "0675aade2351435060878966d4be0572ffac430f9a3166b6c13a657a9dbbd731",
-         "bytes_per_launch": {"c5_llada_l4096_b8": 552370000}}],
+         "sha256": "bfec166c49fcaea673858dc2e86bfa2b1bffe4d191e2c41857dac13d2d180d5a",
+         "bytes_per_launch": {"c5_llada_l4096_b8": 552480000}}],
     "attend_dense": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
-         "sha256": "9633a97b1fa145586220abd4f95827e8d6e35f1c6512fcb5089beec8b73980a4",
-         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62860000, "c5_llada_l4096": 163660000}}],
+         "sha256": "ca69a0676523b22b75dfd9c70e8a3f9e7d9b0590a281e176eada860b6ef54d03",
+         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 64550000, "c5_llada_l4096": 161680000}}],
     "entropy_gate": [
         {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
          "sha256": "9aff17035d14500e5378489b0f9cb64e1b4f42fbe658d39056e2c7edeb701d42",
