@@ -74,7 +74,17 @@ typedef struct {
     int32_t head_dim;    /* D: 64 or 128 */
     int32_t dtype;       /* ec_dtype of q, k_new, v_new, the caches and out */
     float   scale;       /* softmax scale; 0 means 1/sqrt(head_dim) */
+    uint32_t flags;      /* EC_ATTN_* bits; 0 is always correct */
 } ec_attn_desc;
+
+/* (No counterpart in the paper: a scheduling permission.)  The caller states that no work still in flight on the
+ * stream when ec_attend starts writes k_cache or v_cache -- typically the kernel enqueued right before the call is
+ * the projection that produced q, k_new and v_new, or the attention of another layer with caches of its own.  The
+ * kernels are launched with programmatic stream serialisation; with this bit they may ask for cached K/V tiles
+ * before they wait for the preceding kernel to finish (q, k_new, v_new and active_idx are always read after that
+ * wait).  Do not set it when the preceding work on the stream may still be writing these caches, e.g. an
+ * ec_kv_refresh or ec_attend on the same caches enqueued immediately before. */
+#define EC_ATTN_CACHE_SETTLED 1u
 
 /* Layouts
  *   k_cache, v_cache  [batch, n_kv_heads, ctx_len, head_dim]

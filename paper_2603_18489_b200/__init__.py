@@ -26,6 +26,7 @@ LIB_PATH = os.path.join(_HERE, "libentropycache.so")
 
 EC_F32, EC_BF16 = 0, 1
 EC_SKIP, EC_RECOMPUTE = 0, 1
+EC_ATTN_CACHE_SETTLED = 1   # ec_attn_desc.flags: nothing in flight on the stream writes the caches
 EC_OK = 0
 
 
@@ -39,7 +40,7 @@ class ec_attn_desc(ctypes.Structure):
     """Mirror of the C struct ec_attn_desc."""
     _fields_ = [("batch", ctypes.c_int32), ("ctx_len", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
                 ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("scale", ctypes.c_float)]
+                ("scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -122,9 +123,9 @@ def _stream(stream) -> ctypes.c_void_p:
 
 
 def make_desc(batch: int, ctx_len: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype,
-              scale: float = 0.0) -> ec_attn_desc:
+              scale: float = 0.0, flags: int = 0) -> ec_attn_desc:
     code = dtype if isinstance(dtype, int) else (EC_BF16 if dtype == torch.bfloat16 else EC_F32)
-    return ec_attn_desc(batch, ctx_len, n_q_heads, n_kv_heads, head_dim, code, scale)
+    return ec_attn_desc(batch, ctx_len, n_q_heads, n_kv_heads, head_dim, code, scale, flags)
 
 
 def desc_from_tensors(q: torch.Tensor, k_cache: torch.Tensor, scale: float = 0.0) -> ec_attn_desc:

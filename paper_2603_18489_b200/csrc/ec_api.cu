@@ -83,6 +83,7 @@ ec_status check_desc(const ec_attn_desc* d) {
     if (d->n_q_heads % d->n_kv_heads != 0) return EC_ERR_SHAPE;
     if (d->head_dim != 64 && d->head_dim != 128) return EC_ERR_UNSUPPORTED;
     if (!(d->scale >= 0.f) || d->scale > 1.0e30f) return EC_ERR_SHAPE;  // also rejects NaN
+    if (d->flags & ~(uint32_t)EC_ATTN_CACHE_SETTLED) return EC_ERR_UNSUPPORTED;   // unknown bits
     return EC_OK;
 }
 

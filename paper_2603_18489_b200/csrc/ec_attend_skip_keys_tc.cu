@@ -27,11 +27,12 @@
 //            that the memory system always has requests queued while the first tiles are consumed;
 //   refresh  the active rows' fresh K/V reach the attention straight from k_new / v_new, not through the cache: one
 //            CTA of every cluster (the last) attends to them as one or two EXTRA key tiles, fetched by TMA from the
-//            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) before its cache
-//            tiles, while every CTA masks the stale cached keys of the refreshed positions (a bit per key, built from
+//            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) after its cache
+//            tiles (visited first they held a ring stage through the start of the stream and set that CTA two tile
+//            times behind its peers), while every CTA masks the stale cached keys of the refreshed positions (a bit per key, built from
 //            the index list).  The attention therefore never waits for the cache update: the auxiliary warps of that
-//            CTA send the fresh rows from the landed tile to the cache in global memory, one TMA row store per row
-//            and half, for later steps, ordered against nothing.  (Keys
+//            CTA copy the fresh rows from the landed tile to the cache in global memory with plain 16-byte stores,
+//            for later steps, ordered against nothing.  (Keys
 //            in a different order, the same sum.)  When a CTA holds a single cache tile the extra tiles get a CTA of
 //            their own, so that nobody streams two tiles through one stage;
 //   merge    CTA c of the cluster owns the output columns d in [c*DL, (c+1)*DL): once every CTA of the cluster is
@@ -67,7 +68,7 @@ constexpr int kMaxActive = 256;            // active rows of a sequence (refresh
 constexpr int kMaxTiles = 1024;            // key tiles of one CTA (bits of the patch mask)
 
 enum { B_FULL = 0, B_EMPTY = kMaxStages, B_SFULL = 2 * kMaxStages, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 1,
-       B_PSUM = B_PVDONE + 1, B_QFULL = B_PSUM + 1, B_LIST = B_QFULL + 1, B_FRESHOUT = B_LIST + 1, B_RECV = B_FRESHOUT + 2,
+       B_PSUM = B_PVDONE + 1, B_QFULL = B_PSUM + 1, B_LIST = B_QFULL + 1, B_RECV = B_LIST + 1,
        B_COUNT = B_RECV + 1 };
 
 constexpr uint32_t kBarBytes = (B_COUNT * 8u + 15u) & ~15u;   // the barrier block, padded so that what follows is 16-byte aligned
@@ -130,6 +131,9 @@ struct KeysParams {
     // the first fill of its ring by this much per stage, so that the stages of the launch arrive one wave after the
     // other instead of all together (0: no spacing).
     uint32_t stagger_ns;
+    // 1: the caller stated (EC_ATTN_CACHE_SETTLED) that nothing still running on the stream writes the caches, so the
+    // first cache tile is asked for before the dependency wait
+    int early_cache;
 };
 
 // words after the barrier block
@@ -150,8 +154,7 @@ template <int N>
 __global__ void __launch_bounds__(64 + (N > 64 ? 256 : 128) + kAuxThreads, N <= 64 ? 2 : 1)
 attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kn,
-                        const __grid_constant__ CUtensorMap map_vn, const __grid_constant__ CUtensorMap map_k1,
-                        const __grid_constant__ CUtensorMap map_v1, const KeysParams p) {
+                        const __grid_constant__ CUtensorMap map_vn, const KeysParams p) {
     static_assert(N == 48 || N == 64 || N == 96, "query-row slots per CTA");
     constexpr int WG = N > 64 ? 2 : 1;          // softmax warpgroups: each takes NH of a key's N scores
     constexpr int NH = N / WG;
@@ -186,7 +189,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int TC = max(0, t_end - t_begin);                  // cache tiles of this CTA
     const int NS = p.n_stages;
     const bool refresh = p.k_new != nullptr;
-    // the last CTA of the cluster attends to the fresh rows first, as XT extra key tiles read from k_new / v_new
+    // the last CTA of the cluster attends to the fresh rows too, after its cache tiles, as XT extra key tiles read from
+    // k_new / v_new: visits [0, TC) are cache tiles, visits [TC, T) fresh tiles
     const int XT = (refresh && split == p.n_splits - 1) ? p.n_extra : 0;
     const int T = XT + TC;           // tiles this CTA visits: >= 1 by construction of the plan
     const int key_lo = t_begin * BK, key_hi = min(p.ctx_len, t_end * BK);
@@ -197,25 +201,37 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const uint32_t chunk_bytes = chunk_floats * 4u;
     const uint32_t stg_off = 0, recv_off = (uint32_t)C * chunk_bytes;
 
-    // ---- set-up (touches no global memory) -------------------------------------------------
+    // ---- set-up ------------------------------------------------------------------------------
+    // Under programmatic dependent launch this CTA starts while the tail of the previous kernel still runs.  Whatever
+    // that kernel produces (q, k_new, v_new, the index list) is read after the dependency wait below.  The caches are
+    // read before it only when the caller has stated that nothing in flight writes them: the producer thread then asks
+    // for its first cache tile as soon as the barriers exist, and the memory system works through the rest of the
+    // set-up, the previous kernel's tail and the wait.
+    unsigned long long t_fill = 0;
     if (tid == 0) {
-        prefetch_map(&map_k);
-        prefetch_map(&map_v);
-        if (p.q_tma) prefetch_map(&map_q);
-        if (p.k_new) {
-            prefetch_map(&map_kn);
-            prefetch_map(&map_vn);
-            prefetch_map(&map_k1);
-            prefetch_map(&map_v1);
-        }
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1;
             if (i == B_PFULL || (i == B_QFULL && !p.q_tma)) count = kSoft;
-            if (i == B_PSUM || i == B_FRESHOUT || i == B_FRESHOUT + 1) count = kAuxThreads;
+            if (i == B_PSUM) count = kAuxThreads;
             mbar_init(bar(i), count);
         }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (p.early_cache && TC > 0) {   // ring entry 0: the first cache tile
+            t_fill = global_timer_ns();
+            const uint32_t dst = base + p.off_stage;
+            mbar_expect_tx(bar(B_FULL + 0), STAGE);
+            tma_load_4d(dst, &map_k, 0, t_begin * BK, 0, bh, bar(B_FULL + 0));
+            tma_load_4d(dst + TILE, &map_v, 0, t_begin * BK, 0, bh, bar(B_FULL + 0));
+        } else {
+            prefetch_map(&map_k);
+            prefetch_map(&map_v);
+        }
+        if (p.q_tma) prefetch_map(&map_q);
+        if (p.k_new) {
+            prefetch_map(&map_kn);
+            prefetch_map(&map_vn);
+        }
         if (C > 1) mbar_expect_tx(bar(B_RECV), (uint32_t)C * chunk_bytes);   // the peers' partials, one chunk each
     }
     if (tid < kMaxTiles / 32) sh->patch_mask[tid] = 0u;
@@ -239,27 +255,28 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 mbar_expect_tx(bar(B_QFULL), (uint32_t)N * 256u);
                 tma_load_5d(base, &map_q, 0, i0, hq0, 0, b, bar(B_QFULL));   // rows past the chunk land in unused slots
             }
-            const unsigned long long t_fill = global_timer_ns();
+            const bool first_asked = t_fill != 0;   // ring entry 0 (the first cache tile) is already on its way
+            if (!first_asked) t_fill = global_timer_ns();
             for (int j = 0; j < T; ++j) {
                 const int s = j % NS, u = j / NS;
-                if (u == 0 && j > XT && p.stagger_ns) {
+                if (first_asked && j == 0) continue;
+                if (u == 0 && j > 0 && j < TC && p.stagger_ns) {
                     // First fill of the ring: cache stage c of every CTA is asked for c * stagger_ns after the first, so
                     // the first tiles of all CTAs land before anybody's second, and requests stay queued while they
                     // are consumed.  (Asked for all at once, the stages of the whole launch arrive together after
                     // the time of all of them, and the memory system then idles until the first stage is free again.)
-                    const unsigned long long due = t_fill + (unsigned long long)(j - XT) * p.stagger_ns;
+                    const unsigned long long due = t_fill + (unsigned long long)j * p.stagger_ns;
                     while (global_timer_ns() < due) __nanosleep(64);
                 }
                 if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
-                if (u > 0 && j - NS < XT && sub == 0)   // the stage held a fresh tile: the cache update has read it
-                    mbar_wait(bar(B_FRESHOUT + (j - NS)), 0, abort_flag, p.dev_status);   // (one single-phase barrier per fresh tile)
                 const uint32_t dst = base + p.off_stage + s * STAGE;
                 mbar_expect_tx(bar(B_FULL + s), STAGE);
-                if (j < XT) {   // active rows [128 j, 128 j + 128) of this kv head, fresh; rows past n_active read as zero
-                    tma_load_5d(dst, &map_kn, 0, j * BK, 0, hk, b, bar(B_FULL + s));
-                    tma_load_5d(dst + TILE, &map_vn, 0, j * BK, 0, hk, b, bar(B_FULL + s));
+                if (j >= TC) {   // active rows [128 x, 128 x + 128) of this kv head, fresh; rows past n_active read as zero
+                    const int x = j - TC;
+                    tma_load_5d(dst, &map_kn, 0, x * BK, 0, hk, b, bar(B_FULL + s));
+                    tma_load_5d(dst + TILE, &map_vn, 0, x * BK, 0, hk, b, bar(B_FULL + s));
                 } else {
-                    const int key0 = (t_begin + j - XT) * BK;
+                    const int key0 = (t_begin + j) * BK;
                     tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
                     tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
                 }
@@ -362,39 +379,6 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     } else if (warp >= 2 + 4 * WG) {
         // ===== auxiliary warps: the fresh rows into the cache (for later steps); row sums of P^T =====
         const int atid = tid - (64 + kSoft);
-        if (XT > 0 && sub == 0) {
-            // One CTA per (sequence, kv head) -- the one that attends to the fresh tiles -- also puts the active rows'
-            // K/V into the cache, for later steps: the fresh tile is in shared memory already, so each row leaves as four
-            // TMA stores of 128 bytes (K and V, two 64-column halves) to its position in the cache.  Nothing in this launch
-            // depends on these stores; the producer only waits until they have read the tile before it refills the stage.
-            int posx[2];
-#pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {   // positions of this thread's rows of the first fresh tile, fetched ahead
-                const int i = rr * kAuxThreads + atid;
-                posx[rr] = (i < p.n_active) ? (p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i) : -1;
-            }
-            for (int x = 0; x < XT; ++x) {
-                mbar_wait(bar(B_FULL + x % NS), (x / NS) & 1, abort_flag, p.dev_status);   // the fresh tile has landed
-                const uint32_t tile = base + p.off_stage + (x % NS) * STAGE;
-#pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const int r = rr * kAuxThreads + atid, i = x * BK + r;
-                    int pos = posx[rr];
-                    if (x > 0) pos = (i < p.n_active) ? (p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i) : -1;
-                    if (pos >= 0 && pos < p.ctx_len) {
-                        const uint32_t row = tile + (r >> 3) * 1024 + (r & 7) * 128;
-                        tma_store_4d(&map_k1, 0, pos, 0, bh, row);
-                        tma_store_4d(&map_k1, 0, pos, 1, bh, row + SUB);
-                        tma_store_4d(&map_v1, 0, pos, 0, bh, row + TILE);
-                        tma_store_4d(&map_v1, 0, pos, 1, bh, row + TILE + SUB);
-                    }
-                }
-                bulk_commit();
-                bulk_wait_read();
-                mbar_arrive(bar(B_FRESHOUT + x));
-            }
-        }
-
         // row sums: this thread adds up column pair cp of the keys [k_lo, k_lo + BK / kParts) of every tile
         const bool summer = atid < kPairs * kParts;
         const int cp = atid % kPairs, col = 2 * cp, gch = col >> 3;
@@ -403,6 +387,29 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         float acc0 = 0.f, acc1 = 0.f;
 
         for (int j = 0; j < T; ++j) {
+            if (j >= TC && sub == 0) {
+                // One CTA per (sequence, kv head) -- the one that attends to the fresh tiles -- also puts the active
+                // rows' K/V into the cache, for later steps: the fresh tile is in shared memory once its stage is full,
+                // so the rows leave from there as plain 16-byte stores (thread = one 16-byte piece of a row, four rows
+                // per pass; the tile is 128-byte swizzled).  Nothing in this launch depends on these stores.  The stage
+                // is overwritten (by the merge's exchange areas) only after the row sums of the last visit, which this
+                // thread reports after it has read its pieces.  (One TMA store per row and half took 3.5 us for 34
+                // rows: 136 requests of 128 bytes, served one after the other.)
+                const int x = j - TC;
+                mbar_wait(bar(B_FULL + j % NS), (j / NS) & 1, abort_flag, p.dev_status);   // the fresh tile has landed
+                const unsigned char* tile = gbase + p.off_stage + (j % NS) * STAGE;
+                const int ch = atid & 15;   // piece of the row: columns [8 ch, 8 ch + 8)
+                const int n_rows = min(BK, p.n_active - x * BK);
+                for (int r = atid >> 4; r < n_rows; r += kAuxThreads / 16) {
+                    const int i = x * BK + r;
+                    const int pos = p.active_idx ? __ldg(p.active_idx + (long long)b * p.n_active + i) : i;
+                    if (pos < 0 || pos >= p.ctx_len) continue;
+                    const uint32_t off = (ch >> 3) * SUB + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4);
+                    const long long dst = (((long long)bh * p.ctx_len + pos) * HD + ch * 8);
+                    *reinterpret_cast<uint4*>(p.k_cache + dst) = *reinterpret_cast<const uint4*>(tile + off);
+                    *reinterpret_cast<uint4*>(p.v_cache + dst) = *reinterpret_cast<const uint4*>(tile + TILE + off);
+                }
+            }
             // P^T of tile j is in shared memory
             mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.dev_status);
             if (summer) {
@@ -477,10 +484,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             // this thread's key does not count: a missing row of a fresh tile, a key past the end of the context (ragged
             // last tile), a cached key whose position is being refreshed (it is attended from the fresh tile instead)
             bool past_end;
-            if (j < XT) {
-                past_end = !((fresh_ok >> j) & 1u);
+            if (j >= TC) {
+                past_end = !((fresh_ok >> (j - TC)) & 1u);
             } else {
-                const int t = j - XT;
+                const int t = j;
                 past_end = (t_begin + t) * BK + kk >= p.ctx_len;
                 if (!masks_ready) {
                     mbar_wait(bar(B_LIST), 0, abort_flag, p.dev_status);
@@ -699,20 +706,6 @@ bool make_cache_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// the same cache as the target of the refresh: boxes of one key and one 64-column half (128 bytes), so that a row of a
-// tile in shared memory can be stored to an arbitrary position
-bool make_cache_row_map(CUtensorMap* map, const void* cache, int bh, int ctx_len) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[4] = {64, (cuuint64_t)ctx_len, 2, (cuuint64_t)bh};
-    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)ctx_len * HD * 2};
-    const cuuint32_t box[4] = {64, 1, 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(cache), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // q [B, n, H_q, 128] bf16 (one query head per CTA column) seen as 5-D {64 columns, row, head, half, sequence}:
 // the box {64, N, 1, 2, 1} lands as [half][row][64 columns], the K-major Q tile; rows past n read as zero
 bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_q_heads, int n_slots) {
@@ -918,8 +911,8 @@ double stream_bytes_per_ns() {
 
 template <int N>
 cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap& mk, const CUtensorMap& mv,
-                     const CUtensorMap& mq, const CUtensorMap& mkn, const CUtensorMap& mvn, const CUtensorMap& mk1,
-                     const CUtensorMap& mv1, int bh, cudaStream_t stream) {
+                     const CUtensorMap& mq, const CUtensorMap& mkn, const CUtensorMap& mvn,
+                     int bh, cudaStream_t stream) {
     static PerDeviceOnce attr_once;
     if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_skip_keys_kernel<N>, (int)kSmemMax); ea != cudaSuccess)
         return ea;
@@ -937,7 +930,7 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, mq, mkn, mvn, mk1, mv1, p);
+    return cudaLaunchKernelEx(&cfg, attend_skip_keys_kernel<N>, mk, mv, mq, mkn, mvn, p);
 }
 
 }  // namespace
@@ -970,12 +963,11 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     if (!make_cache_map(&map_k, a.k_cache, bh, a.d.ctx_len) || !make_cache_map(&map_v, a.v_cache, bh, a.d.ctx_len))
         return cudaErrorInvalidValue;
     KeysParams p{};
-    CUtensorMap map_q = map_k, map_kn = map_k, map_vn = map_v, map_k1 = map_k, map_v1 = map_v;   // placeholders unless q_tma / fresh
+    CUtensorMap map_q = map_k, map_kn = map_k, map_vn = map_v;   // placeholders unless q_tma / fresh
     p.q_tma = (pl.group == 1) ? 1 : 0;   // one query head per CTA column: its rows are one TMA box
     if (p.q_tma && !make_q_map(&map_q, a.q, a.d.batch, a.n_active, a.d.n_q_heads, pl.n_slots)) return cudaErrorInvalidValue;
     if (fresh && (!make_fresh_map(&map_kn, k_new, a.d.batch, a.n_active, a.d.n_kv_heads) ||
-                  !make_fresh_map(&map_vn, v_new, a.d.batch, a.n_active, a.d.n_kv_heads) ||
-                  !make_cache_row_map(&map_k1, a.k_cache, bh, a.d.ctx_len) || !make_cache_row_map(&map_v1, a.v_cache, bh, a.d.ctx_len)))
+                  !make_fresh_map(&map_vn, v_new, a.d.batch, a.n_active, a.d.n_kv_heads)))
         return cudaErrorInvalidValue;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
@@ -1003,6 +995,7 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.off_list = pl.off_list;
     p.off_bar = pl.off_bar;
     p.scale_log2 = a.scale * kLog2e;
+    p.early_cache = (a.d.flags & EC_ATTN_CACHE_SETTLED) ? 1 : 0;
     p.stagger_ns = 0;
     if (pl.tiles_per_split > 1) {
         const double streams = (double)pl.n_splits * bh;   // CTAs with K/V of their own (columns of one head share it through L2)
@@ -1010,9 +1003,9 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
         p.stagger_ns = (uint32_t)(ns < 3000.0 ? ns : 3000.0);
     }
     const int cols = bh * pl.n_sub;
-    return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)
-           : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream)
-                              : launch_n<96>(pl, p, map_k, map_v, map_q, map_kn, map_vn, map_k1, map_v1, cols, stream);
+    return pl.n_slots == 48   ? launch_n<48>(pl, p, map_k, map_v, map_q, map_kn, map_vn, cols, stream)
+           : pl.n_slots == 64 ? launch_n<64>(pl, p, map_k, map_v, map_q, map_kn, map_vn, cols, stream)
+                              : launch_n<96>(pl, p, map_k, map_v, map_q, map_kn, map_vn, cols, stream);
 }
 
 }  // namespace ec

@@ -206,3 +206,44 @@ def test_few_row_skip_step_with_rising_maxima():
     k = k + ramp * q.mean(axis=1)[:, :, None, :] * 8.0
     t["k_cache"] = syn.encode(k.astype(np.float32), syn.BF16)
     _check(w, t, scale=1.0, refresh=False)
+
+
+@pytest.mark.parametrize("name,n_layers", [("c4_llada_l2048", 4), ("c3_dream_l768", 3), ("c2_llada_l768", 4)])
+def test_back_to_back_layers_with_the_cache_settled_flag(name, n_layers):
+    """EC_ATTN_CACHE_SETTLED lets a launch ask for cached tiles before the previous kernel of the stream has finished.
+    Three passes over `n_layers` layers with caches of their own, enqueued back to back with no synchronisation (the
+    situation the flag describes: the kernel before a launch works on another layer's caches); every pass refreshes
+    different rows, so a launch that read a cache before its own earlier refresh had landed, or a refresh lost to
+    the overlap, shows up in the outputs of the later passes or in the final cache bytes."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.WORKLOADS[name]
+    n = w.n_skip_rows
+    d = ec.make_desc(w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, flags=ec.EC_ATTN_CACHE_SETTLED)
+    assert ec.ec_attend_kernel_name(d, n, True, True).startswith("attend_skip_keys_kernel")
+    n_pass = 3
+    ins = [[syn.attn_inputs(w, n, step=p, salt=50 + l, block_no=p) for l in range(n_layers)] for p in range(n_pass)]
+    kc = [ins[0][l]["k_cache"].copy() for l in range(n_layers)]
+    vc = [ins[0][l]["v_cache"].copy() for l in range(n_layers)]
+    gk = [to_dev(kc[l]) for l in range(n_layers)]
+    gv = [to_dev(vc[l]) for l in range(n_layers)]
+    dev = [[{k: to_dev(ins[p][l][k]) for k in ("q", "k_new", "v_new", "active_idx")} for l in range(n_layers)]
+           for p in range(n_pass)]
+    outs = [[torch.empty_like(dev[p][l]["q"]) for l in range(n_layers)] for p in range(n_pass)]
+    ws = ec.new_workspace(max(16, ec.ec_attend_workspace_bytes(d, n)))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    for p in range(n_pass):
+        for l in range(n_layers):
+            t = dev[p][l]
+            ec.ec_attend(d, t["q"], t["k_new"], t["v_new"], gk[l], gv[l], t["active_idx"], out=outs[p][l],
+                         workspace=ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for p in range(n_pass):
+        for l in range(n_layers):
+            t = ins[p][l]
+            ref = oracle.refresh_and_attend(t["q"], t["k_new"], t["v_new"], kc[l], vc[l], t["active_idx"], w.dtype)
+            assert np.abs(to_f64(outs[p][l]) - ref).max() <= BF16_TOL, (p, l)
+    for l in range(n_layers):
+        assert np.array_equal(to_storage(gk[l]), kc[l]) and np.array_equal(to_storage(gv[l]), vc[l])
