@@ -55,8 +55,8 @@ K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dr
 NCU_TRAFFIC = {
     "attend_skip": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-         "sha256": "4e4c7fc5a90767439edacee25758e74549d67d3e91ef33574a4fd8ca09109af3",
-         "bytes_per_launch": {"c2_llada_l768": 13510000, "c5_llada_l4096": 68160000}},
+         "sha256": "56358dbda13ef444eae93ef1111ad7fa45d20efc64d2a78e4774ac8a6b877f89",
+         "bytes_per_launch": {"c2_llada_l768": 13500000, "c5_llada_l4096": 68670000}},
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
          "sha256": "bfec166c49fcaea673858dc2e86bfa2b1bffe4d191e2c41857dac13d2d180d5a",
          "bytes_per_launch": {"c5_llada_l4096_b8": 552480000}}],
