@@ -59,6 +59,8 @@ size_t attend_ws(const ec_attn_desc& d, int n_active) {
     if (d.dtype == EC_BF16 && d.head_dim == 128) {
         const size_t t = attend_tc_workspace_bytes(d, n_active);
         if (t > n) n = t;
+        const size_t dn = attend_dense_workspace_bytes(d, n_active);
+        if (dn > n) n = dn;
     }
     return n;
 }

@@ -74,7 +74,13 @@ struct DenseParams {
     // those of the real kv head h / kv_div, of which there are n_kv_real.  kv_div = 1 otherwise.
     int kv_div, n_kv_real;
     float scale_log2;
+    // Launch order = unit order (row-tile pair fastest, then head).  The first n_full units are whole; each later
+    // unit (the last, partial wave of the launch) is cut along the keys into `split` CTAs that leave un-normalised
+    // partials in the workspace for combine_cut_units_kernel.  split = 1: no cuts.
+    int n_pairs, n_full, split;
+    float* part;      // [cut unit][part][row tile][128 rows x 128 floats, then m[128], then l[128]]
 };
+constexpr int kPartFloats = BM * (HD + 2);   // one row tile of one part
 
 __global__ void __launch_bounds__(kThreads, 1)
 attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -93,11 +99,18 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pair = blockIdx.x, bh = blockIdx.y;
+    const int lin = blockIdx.x;
+    const bool cut = lin >= p.n_full;
+    const int unit = cut ? p.n_full + (lin - p.n_full) / p.split : lin;
+    const int part = cut ? (lin - p.n_full) % p.split : 0;
+    const int pair = unit % p.n_pairs, bh = unit / p.n_pairs;
     const int b = bh / p.n_kv_heads, hk = bh % p.n_kv_heads;
     const int r_pair = pair * 2 * BM;
     const int n_tiles_q = (p.rows_total - r_pair > BM) ? 2 : 1;   // row tiles of this CTA that hold rows
-    const int T = (p.ctx_len + BN - 1) / BN;
+    const int T_all = (p.ctx_len + BN - 1) / BN;
+    const int tiles_per_part = cut ? (T_all + p.split - 1) / p.split : T_all;
+    const int j0 = part * tiles_per_part;                        // first key tile of this CTA
+    const int T = min(T_all, j0 + tiles_per_part) - j0;          // >= 1 by construction of the plan
 
     if (tid == 0) {
         prefetch_map(&map_k);
@@ -132,7 +145,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 const int slot = n % kSlots, u = n / kSlots;
                 if (u > 0) mbar_wait(bar(B_EMPTY + slot), (u - 1) & 1, abort_flag, p.dev_status);
                 mbar_expect_tx(bar(B_FULL + slot), TILE);
-                tma_load_5d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (n >> 1) * BN, 0, hk_kv, b, bar(B_FULL + slot));
+                tma_load_5d(base + OFF_RING + slot * TILE, (n & 1) ? &map_v : &map_k, 0, (j0 + (n >> 1)) * BN, 0, hk_kv, b, bar(B_FULL + slot));
             }
         }
     } else if (warp == 1) {
@@ -199,7 +212,7 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 ld32(tm_s + h * 64, sr);
                 ld32(tm_s + h * 64 + 32, sr + 32);
                 wait_ld();
-                const int key0 = j * BN + h * 64;
+                const int key0 = (j0 + j) * BN + h * 64;
                 if (key0 + 64 > p.ctx_len) {
 #pragma unroll
                     for (int c = 0; c < 64; ++c)
@@ -260,44 +273,70 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                 mbar_arrive(bar(B_PFULL + t));
             }
 
-            // ---- epilogue: normalise and store this thread's 64 columns ---------------------------
+            // ---- epilogue ------------------------------------------------------------------------
             mbar_wait(bar(B_PVDONE + t), (T - 1) & 1, abort_flag, p.dev_status);
             fence_after();
             *xch_mine = l_run;
             named_barrier(pair_bar, 64);
-            const float inv = 1.f / (l_run + *xch_other);
+            const float l_row = l_run + *xch_other;   // both halves of a row carry the same reference maximum
             const bool valid = r < p.rows_total;
             const int i = valid ? r / p.group : 0, jh = valid ? r % p.group : 0;
             __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hk * p.group + jh) * HD + h * 64;
+            if (!cut) {
+                // whole unit: normalise and store this thread's 64 columns
+                const float inv = 1.f / l_row;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t o[32];
-                ld32(tm_o + h * 64 + c * 32, o);
-                wait_ld();
-                if (valid && !*abort_flag) {   // a CTA whose wait gave up stores nothing
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+                    ld32(tm_o + h * 64 + c * 32, o);
+                    wait_ld();
+                    if (valid && !*abort_flag) {   // a CTA whose wait gave up stores nothing
 #pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
-                        w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
-                        w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
-                        w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
+                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
+                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
+                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
+                        }
                     }
+                }
+            } else {
+                // part of a cut unit: the un-normalised row (relative to m_used), m and l go to the workspace; the
+                // combine kernel that follows in the stream merges the parts (one CTA combining a unit on its own is
+                // bound by what a single SM can pull out of L2: 11 us per extra part)
+                const int cu = unit - p.n_full;
+                float* mine = p.part + ((size_t)(cu * p.split + part) * 2 + t) * kPartFloats;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+                    ld32(tm_o + h * 64 + c * 32, o);
+                    wait_ld();
+                    if (!*abort_flag) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 8; ++v4)
+                            *reinterpret_cast<uint4*>(mine + row * HD + h * 64 + c * 32 + v4 * 4) =
+                                make_uint4(o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
+                    }
+                }
+                if (h == 0 && !*abort_flag) {
+                    mine[BM * HD + row] = m_used;
+                    mine[BM * HD + BM + row] = l_row;
                 }
             }
         }
         fence_before();
-    } else if (p.k_dst != nullptr) {
+    } else if (p.k_dst != nullptr && part == 0) {
         // ====================== copy warp: this CTA's share of the refresh ============================
         // The (row-tile pair, kv head) CTAs of a head split its positions evenly; a position's K and V rows
         // (256 bytes each) go from [b, pos, hk, :] to [b, hk, pos, :].  Two rows per warp instruction, eight
         // instructions in flight.  Nobody reads the cache in this launch.
         // (with one unit per query head, the kv_div units of a real kv head share its positions as well)
         const int hk_kv = hk / p.kv_div;
-        const int n_share = gridDim.x * p.kv_div;
+        const int n_share = p.n_pairs * p.kv_div;
         const int per = (p.ctx_len + n_share - 1) / n_share;
-        const int pos0 = ((hk % p.kv_div) * gridDim.x + pair) * per, pos1 = min(p.ctx_len, pos0 + per);
+        const int pos0 = ((hk % p.kv_div) * p.n_pairs + pair) * per, pos1 = min(p.ctx_len, pos0 + per);
         const int sub = lane >> 4, piece = lane & 15;
         for (int pos = pos0; pos < pos1; pos += 16) {
             uint4 kv[8], vv[8];
@@ -329,6 +368,68 @@ attend_dense_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     }
 }
 
+// Merges the parts of the cut units: CTA = 32 rows of one row tile of one cut unit, thread = 16 columns of a row.
+// With M the largest reference maximum of the row's parts and w_q = 2^(m_q - M):  out = sum_q w_q O_q / sum_q w_q l_q.
+struct CombineParams {
+    const float* part;
+    __nv_bfloat16* out;
+    int n_pairs, n_full, split, n_active, n_q_heads, rows_total;
+};
+__global__ void __launch_bounds__(256) combine_cut_units_kernel(const CombineParams p) {
+    pdl_wait();   // the partials of the attention launch are complete
+    pdl_launch_dependents();
+    const int cu = blockIdx.x >> 3, t = (blockIdx.x >> 2) & 1, row = (blockIdx.x & 3) * 32 + (threadIdx.x >> 3);
+    const int c0 = (threadIdx.x & 7) * 16;
+    const int unit = p.n_full + cu;
+    const int pair = unit % p.n_pairs, bh = unit / p.n_pairs;
+    const int b = bh / p.n_q_heads, hq = bh % p.n_q_heads;
+    const int r = pair * 2 * BM + t * BM + row;
+    if (r >= p.rows_total) return;
+    float w[8], M = -INFINITY, L = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        w[q] = -INFINITY;
+        if (q < p.split) {
+            w[q] = __ldcg(p.part + ((size_t)(cu * p.split + q) * 2 + t) * kPartFloats + BM * HD + row);
+            M = fmaxf(M, w[q]);
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (q < p.split) {
+            w[q] = fast_exp2(w[q] - M);
+            L = fmaf(w[q], __ldcg(p.part + ((size_t)(cu * p.split + q) * 2 + t) * kPartFloats + BM * HD + BM + row), L);
+        }
+    }
+    float acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (q < p.split) {
+            const float4* src = reinterpret_cast<const float4*>(
+                p.part + ((size_t)(cu * p.split + q) * 2 + t) * kPartFloats + row * HD + c0);
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+                const float4 f = __ldcg(src + v4);
+                acc[v4 * 4 + 0] = fmaf(w[q], f.x, acc[v4 * 4 + 0]);
+                acc[v4 * 4 + 1] = fmaf(w[q], f.y, acc[v4 * 4 + 1]);
+                acc[v4 * 4 + 2] = fmaf(w[q], f.z, acc[v4 * 4 + 2]);
+                acc[v4 * 4 + 3] = fmaf(w[q], f.w, acc[v4 * 4 + 3]);
+            }
+        }
+    }
+    const float inv = 1.f / L;
+    __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + r) * p.n_q_heads + hq) * HD + c0;
+    uint4 o0, o1;
+    o0.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);   o0.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+    o0.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);   o0.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+    o1.x = pack_bf16x2(acc[8] * inv, acc[9] * inv);   o1.y = pack_bf16x2(acc[10] * inv, acc[11] * inv);
+    o1.z = pack_bf16x2(acc[12] * inv, acc[13] * inv); o1.w = pack_bf16x2(acc[14] * inv, acc[15] * inv);
+    *reinterpret_cast<uint4*>(dst) = o0;
+    *reinterpret_cast<uint4*>(dst + 8) = o1;
+}
+
 // ---- host side ---------------------------------------------------------------------------
 // Q of an MHA step seen as 5-D {64 columns, active row, head, half, sequence}: one box {64, 128, 1, 2, 1} lands as the
 // two 128-byte-swizzled halves of a [128 rows x 128] tile; rows past n_active read as zero.
@@ -350,25 +451,69 @@ bool make_kv_map(CUtensorMap* map, const void* ptr, int batch, int n_kv_heads, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// How the launch is cut.  Units = (sequence, query head, row-tile pair); a unit walks over all T key tiles.  The
+// hardware deals the CTAs to the SMs in launch order, so the last units form a partial wave: `tail` units on `sms` SMs.
+// Cutting each of them along the keys into s CTAs (s = 2, 4 or 8, at least four key tiles each) fills that wave:
+// cost in key-tile times, with two tiles' worth of fixed cost per CTA, one more for writing the partials, and four
+// for the combine launch that follows:
+//     waves_full * (T + 2) + ceil(tail * s / sms) * (ceil(T / s) + 3) + 4
+// s = 1 (no cut) unless a cut saves at least 3 %.
+struct DensePlan {
+    int n_pairs, units, n_full, split, n_ctas;
+};
+DensePlan make_dense_plan(const ec_attn_desc& d, int n_active) {
+    DensePlan pl;
+    pl.n_pairs = (n_active + 2 * BM - 1) / (2 * BM);
+    pl.units = pl.n_pairs * d.batch * d.n_q_heads;
+    pl.n_full = pl.units;
+    pl.split = 1;
+    const int sms = sm_count();
+    const long long T = (d.ctx_len + BN - 1) / BN;
+    const long long waves_full = pl.units / sms, tail = pl.units % sms;
+    if (tail > 0) {
+        long long best = (waves_full + 1) * (T + 2);
+        const long long need = best - best * 3 / 100;
+        for (int s = 2; s <= 8; s *= 2) {
+            if (T / s < 4) break;
+            const long long cost = waves_full * (T + 2) + ((tail * s + sms - 1) / sms) * ((T + s - 1) / s + 3) + 4;
+            if (cost < best && cost <= need) {
+                best = cost;
+                pl.split = s;
+            }
+        }
+        if (pl.split > 1) pl.n_full = pl.units - (int)tail;
+    }
+    pl.n_ctas = pl.n_full + (pl.units - pl.n_full) * pl.split;
+    return pl;
+}
+
+
 }  // namespace
 
-// the two-tile kernel has no key split: it is used when the (row-tile pair, kv head) units fill the GPU
+// the two-tile kernel is used when its (row-tile pair, head) units fill the GPU
 bool attend_dense_supported(const ec_attn_desc& d, int n_active) {
     if (d.dtype != EC_BF16 || d.head_dim != HD || n_active < 1) return false;
     // one unit per (sequence, query head, row-tile pair): grouped-query shapes are run head by head
     const long long pairs = ((long long)n_active + 2 * BM - 1) / (2 * BM);
     const long long bh = (long long)d.batch * d.n_q_heads;
-    if (bh > 65535 || pairs > 0x7fffffffLL) return false;
+    if (pairs * bh > 0x3fffffffLL) return false;
     return pairs * bh >= sm_count() / 2;
 }
 
+size_t attend_dense_workspace_bytes(const ec_attn_desc& d, int n_active) {
+    if (!attend_dense_supported(d, n_active)) return 0;
+    const DensePlan pl = make_dense_plan(d, n_active);
+    if (pl.split == 1) return 0;
+    return (size_t)(pl.units - pl.n_full) * pl.split * 2 * kPartFloats * sizeof(float);
+}
+
 void attend_dense_describe(const ec_attn_desc& d, int n_active, char* buf, size_t len) {
-    snprintf(buf, len, "attend_dense_kernel grid=(%d,%d) cluster=1", (n_active + 2 * BM - 1) / (2 * BM),
-             d.batch * d.n_q_heads);
+    const DensePlan pl = make_dense_plan(d, n_active);
+    snprintf(buf, len, "attend_dense_kernel grid=(%d,%d) cluster=1 whole_units=%d cut_units=%dx%d", pl.n_pairs,
+             d.batch * d.n_q_heads, pl.n_full, pl.units - pl.n_full, pl.split);
 }
 
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
-    const int bh = a.d.batch * a.d.n_q_heads;
     CUtensorMap map_k, map_v;
     if (!make_kv_map(&map_k, a.k_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major) ||
         !make_kv_map(&map_v, a.v_cache, a.d.batch, a.d.n_kv_heads, a.d.ctx_len, a.kv_token_major))
@@ -391,6 +536,15 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     p.kv_div = a.d.n_q_heads / a.d.n_kv_heads;
     p.n_kv_real = a.d.n_kv_heads;
     p.scale_log2 = a.scale * kLog2e;
+    const DensePlan pl = make_dense_plan(a.d, a.n_active);
+    p.n_pairs = pl.n_pairs;
+    p.n_full = pl.n_full;
+    p.split = pl.split;
+    p.part = nullptr;
+    if (pl.split > 1) {
+        if (!a.workspace || a.workspace_bytes < attend_dense_workspace_bytes(a.d, a.n_active)) return cudaErrorInvalidValue;
+        p.part = static_cast<float*>(a.workspace);
+    }
     CUtensorMap map_q;
     {
         EncodeTiledFn fn = encode_fn();
@@ -408,7 +562,7 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     static PerDeviceOnce attr_once;
     if (const cudaError_t ea = ensure_dynamic_smem(attr_once, attend_dense_kernel, (int)SMEM_BYTES); ea != cudaSuccess) return ea;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((p.rows_total + 2 * BM - 1) / (2 * BM), bh, 1);
+    cfg.gridDim = dim3(pl.n_ctas, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
@@ -417,7 +571,13 @@ cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, attend_dense_kernel, map_k, map_v, map_q, p);
+    if (const cudaError_t el = cudaLaunchKernelEx(&cfg, attend_dense_kernel, map_k, map_v, map_q, p); el != cudaSuccess) return el;
+    if (pl.split == 1) return cudaSuccess;
+    CombineParams c{p.part, p.out, pl.n_pairs, pl.n_full, pl.split, a.n_active, a.d.n_q_heads, a.n_active};
+    cfg.gridDim = dim3((pl.units - pl.n_full) * 8, 1, 1);   // (cut unit, row tile, 32-row group)
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    return cudaLaunchKernelEx(&cfg, combine_cut_units_kernel, c);
 }
 
 }  // namespace ec

@@ -135,6 +135,7 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
                                     cudaStream_t stream);
 // two-row-tile dense path (bf16, head_dim 128): used when its (row-tile pair, kv head) units fill the GPU
 bool attend_dense_supported(const ec_attn_desc& d, int n_active);
+size_t attend_dense_workspace_bytes(const ec_attn_desc& d, int n_active);   // partials of the cut last wave (0: none)
 cudaError_t launch_attend_dense(const AttendArgs& a, cudaStream_t stream);
 size_t attend_tc_workspace_bytes(const ec_attn_desc& d, int n_active);
 cudaError_t launch_attend_bf16_tc(const AttendArgs& a, cudaStream_t stream);   // tcgen05 path (head_dim 128)

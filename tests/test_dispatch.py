@@ -83,4 +83,9 @@ def test_other_instantiations_and_fallbacks_are_reachable():
     assert name(2, 259, 4, 2, 128, syn.BF16, 259, idx=False) == "refresh_kernel + attend_tc_kernel"
     assert name(2, 130, 6, 3, 64, syn.BF16, 17) == "refresh_kernel + attend_mma_kernel"
     assert name(2, 130, 6, 3, 64, syn.F32, 17) == "refresh_kernel + attend_f32_kernel"
+    # the dense kernel cuts the units of its last, partial wave along the keys when that pays (148 SMs assumed)
+    assert "whole_units=444 cut_units=68x2" in name(1, 4096, 32, 32, 128, syn.BF16, 4096, idx=False)
+    assert "whole_units=444 cut_units=4x8" in name(1, 4096, 28, 4, 128, syn.BF16, 4096, idx=False)
+    assert "cut_units=0x1" in name(1, 2048, 32, 32, 128, syn.BF16, 2048, idx=False)
+    assert "cut_units=0x1" in name(8, 4096, 32, 32, 128, syn.BF16, 4096, idx=False)
     assert ec.ec_attend_kernel_name(ec.make_desc(1, 64, 4, 4, 64, syn.F32), 65, True, True) == ""   # rejected

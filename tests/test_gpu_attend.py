@@ -247,3 +247,24 @@ def test_back_to_back_layers_with_the_cache_settled_flag(name, n_layers):
             assert np.abs(to_f64(outs[p][l]) - ref).max() <= BF16_TOL, (p, l)
     for l in range(n_layers):
         assert np.array_equal(to_storage(gk[l]), kc[l]) and np.array_equal(to_storage(gv[l]), vc[l])
+
+
+@pytest.mark.parametrize("name,Hq,Hkv,L,std_qk,cut", [("dream_l4096", 28, 4, 4096, None, "cut_units=4x8"),
+                                                     ("h19_l2048", 19, 19, 2048, 0.35, "cut_units=4x4"),
+                                                     ("h14_l1536", 14, 7, 1536, 0.35, "cut_units=0x1")])
+def test_recompute_step_whose_last_wave_is_cut_along_the_keys(name, Hq, Hkv, L, std_qk, cut):
+    """The dense kernel cuts the units of its last, partial wave along the keys (2, 4 or 8 parts that leave partials
+    in the workspace; the last to arrive combines them).  Sampled query rows of every head, most of them from the row
+    tiles and heads that the cut units hold (the last ones in launch order), with a peaky score law so that the parts
+    of a row end with different reference maxima; the caches must equal the fresh tensors byte for byte."""
+    import paper_2603_18489_b200 as ec
+
+    w = syn.Workload(95, name, syn.BF16, 1, Hq, Hkv, 128, L - 256, 256, 32, 2, 1024)
+    d = ec.make_desc(1, L, Hq, Hkv, 128, syn.BF16)
+    got = ec.ec_attend_kernel_name(d, L, True, False)
+    assert got.startswith("attend_dense_kernel") and cut in got, got
+    t = syn.attn_inputs(w, L, std_qk=std_qk, salt=3)
+    rng = np.random.Generator(np.random.PCG64(L + Hq))
+    rows = sorted(set(rng.choice(L, 10, replace=False).tolist() + rng.choice(np.arange(L // 2, L), 14, replace=False).tolist()
+                      + [0, L - 1]))
+    _check(w, t, row_sel=rows)
