@@ -62,8 +62,8 @@ NCU_TRAFFIC = {
          "bytes_per_launch": {"c5_llada_l4096_b8": 552480000}}],
     "attend_dense": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_dense_tc.cu",
-         "sha256": "ca69a0676523b22b75dfd9c70e8a3f9e7d9b0590a281e176eada860b6ef54d03",
-         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 64550000, "c5_llada_l4096": 161680000}}],
+         "sha256": "4323d044418277f0fa12a7dee721db22bf5b7291e5e7e0507861c74d0b3dd4fe",
+         "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62770000, "c5_llada_l4096": 176240000}}],
     "entropy_gate": [
         {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
          "sha256": "9aff17035d14500e5378489b0f9cb64e1b4f42fbe658d39056e2c7edeb701d42",
