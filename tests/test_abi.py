@@ -99,3 +99,19 @@ def test_binding_refuses_host_tensors():
     x = torch.zeros(1, 8, 1, 64)
     with pytest.raises(ValueError):
         ec.ec_kv_refresh(d, x, x, x, x, None)
+
+
+def test_descriptor_flags_are_validated_and_mirror_the_header():
+    """ec_attn_desc.flags: the one defined bit is accepted, unknown bits make every entry point that takes the
+    descriptor refuse it (host side, nothing launched); the Python mirror has the C struct's size."""
+    import paper_2603_18489_b200 as ec
+
+    text = open(os.path.join(HEADER_DIR, "entropycache.h")).read()
+    assert re.search(r"#define\s+EC_ATTN_CACHE_SETTLED\s+1u", text) and ec.EC_ATTN_CACHE_SETTLED == 1
+    assert ctypes.sizeof(ec.ec_attn_desc) == 32     # seven 4-byte fields and the flags word
+    ok = ec.make_desc(1, 768, 32, 32, 128, ec.EC_BF16, flags=ec.EC_ATTN_CACHE_SETTLED)
+    bad = ec.make_desc(1, 768, 32, 32, 128, ec.EC_BF16, flags=2)
+    assert ec.ec_attend_workspace_bytes(ok, 34) > 0 and ec.ec_attend_kernel_name(ok, 34) != ""
+    assert ec.ec_attend_workspace_bytes(bad, 34) == 0 and ec.ec_attend_kernel_name(bad, 34) == ""
+    st = ec.lib.ec_attend(ctypes.byref(bad), None, None, None, None, None, None, 34, None, None, 0, None, None)
+    assert st == 6                                  # EC_ERR_UNSUPPORTED, before any pointer is looked at
