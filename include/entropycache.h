@@ -130,7 +130,7 @@ ec_status ec_attend(const ec_attn_desc *desc, const void *q, const void *k_new, 
 /* (No counterpart in the paper: a host-only query for tests and reports.)
  * Describes the launch ec_attend would make for this geometry: the kernel's name with its template instantiation,
  * then "grid=(x,y) cluster=c ..." for the tensor-core kernels, e.g. "attend_skip_keys_kernel<48> grid=(4,32)
- * cluster=4 stages=3 smem=...".  with_fresh_kv: k_new/v_new would be given; with_index_list: active_idx would be
+ * cluster=4 ring_slots=6 smem=...".  with_fresh_kv: k_new/v_new would be given; with_index_list: active_idx would be
  * non-NULL.  Touches no device memory and launches nothing.  Returns "" on arguments ec_attend would reject.  The
  * string lives in a thread-local buffer that the next call on the same thread overwrites. */
 const char *ec_attend_kernel_name(const ec_attn_desc *desc, int32_t n_active, int32_t with_fresh_kv,

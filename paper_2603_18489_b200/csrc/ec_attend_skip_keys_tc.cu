@@ -22,9 +22,12 @@
 //            single tile are small enough for two per SM.  With grouped-query attention the query heads of a kv
 //            head are packed into the N axis; when they exceed the slots the heads (and, beyond 96 active rows,
 //            the rows) are spread over n_sub CTA columns that stream the same K/V (L2 serves the repeats);
-//   K/V      the producer warp issues its TMA loads in key order through a ring of NS stages of 64 KB; they depend on
-//            nothing, and the first fill of the ring is spaced in time (one stage of every CTA per interval) so
-//            that the memory system always has requests queued while the first tiles are consumed;
+//   K/V      the producer warp issues its TMA loads in key order through a ring of NS slots of 32 KB (K_0 V_0 K_1 V_1
+//            ...: a K slot is free again as soon as the scores of its tile are computed, a V slot after the second
+//            product, and an odd slot count is possible, which is what lets the 96-slot instantiation keep two and
+//            a half tiles in flight); the loads depend on nothing, and the first fill of the ring is spaced in time
+//            (one tile of every CTA per interval) so that the memory system always has requests queued while the
+//            first tiles are consumed;
 //   refresh  the active rows' fresh K/V reach the attention straight from k_new / v_new, not through the cache: one
 //            CTA of every cluster (the last) attends to them as one or two EXTRA key tiles, fetched by TMA from the
 //            fresh tensors (a [128 rows x 128] box of k_new is laid out exactly like a cache tile) after its cache
@@ -62,7 +65,7 @@ constexpr int kAuxThreads = 64;           // two warps: cache update and row sum
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr uint32_t STAGE = 2 * TILE;       // K tile + V tile: 64 KB
-constexpr int kMaxStages = 3;
+constexpr int kMaxStages = 6;              // ring slots of one tile (32 KB) each
 constexpr int kMaxSlots = 96;              // query slots (packed rows) of one CTA column
 constexpr int kMaxActive = 256;            // active rows of a sequence (refresh list, row chunks)
 constexpr int kMaxTiles = 1024;            // key tiles of one CTA (bits of the patch mask)
@@ -187,7 +190,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int t_begin = split * p.tiles_per_split;
     const int t_end = min(n_tiles_total, t_begin + p.tiles_per_split);
     const int TC = max(0, t_end - t_begin);                  // cache tiles of this CTA
-    const int NS = p.n_stages;
+    const int NS = p.n_stages;       // ring slots: tile j has K in slot 2j mod NS and V in slot (2j + 1) mod NS
     const bool refresh = p.k_new != nullptr;
     // the last CTA of the cluster attends to the fresh rows too, after its cache tiles, as XT extra key tiles read from
     // k_new / v_new: visits [0, TC) are cache tiles, visits [TC, T) fresh tiles
@@ -220,9 +223,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         if (p.early_cache && TC > 0) {   // ring entry 0: the first cache tile
             t_fill = global_timer_ns();
             const uint32_t dst = base + p.off_stage;
-            mbar_expect_tx(bar(B_FULL + 0), STAGE);
+            mbar_expect_tx(bar(B_FULL + 0), TILE);
             tma_load_4d(dst, &map_k, 0, t_begin * BK, 0, bh, bar(B_FULL + 0));
-            tma_load_4d(dst + TILE, &map_v, 0, t_begin * BK, 0, bh, bar(B_FULL + 0));
+            mbar_expect_tx(bar(B_FULL + 1), TILE);
+            tma_load_4d(dst + TILE, &map_v, 0, t_begin * BK, 0, bh, bar(B_FULL + 1));
         } else {
             prefetch_map(&map_k);
             prefetch_map(&map_v);
@@ -257,28 +261,24 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             }
             const bool first_asked = t_fill != 0;   // ring entry 0 (the first cache tile) is already on its way
             if (!first_asked) t_fill = global_timer_ns();
-            for (int j = 0; j < T; ++j) {
-                const int s = j % NS, u = j / NS;
+            for (int n = 0; n < 2 * T; ++n) {   // ring entry n: K of tile n / 2 (even n) or its V (odd n)
+                const int j = n >> 1, s = n % NS, u = n / NS;
                 if (first_asked && j == 0) continue;
-                if (u == 0 && j > 0 && j < TC && p.stagger_ns) {
-                    // First fill of the ring: cache stage c of every CTA is asked for c * stagger_ns after the first, so
+                if (u == 0 && !(n & 1) && j > 0 && j < TC && p.stagger_ns) {
+                    // First fill of the ring: cache tile j of every CTA is asked for j * stagger_ns after the first, so
                     // the first tiles of all CTAs land before anybody's second, and requests stay queued while they
-                    // are consumed.  (Asked for all at once, the stages of the whole launch arrive together after
-                    // the time of all of them, and the memory system then idles until the first stage is free again.)
+                    // are consumed.  (Asked for all at once, the tiles of the whole launch arrive together after
+                    // the time of all of them, and the memory system then idles until the first slot is free again.)
                     const unsigned long long due = t_fill + (unsigned long long)j * p.stagger_ns;
                     while (global_timer_ns() < due) __nanosleep(64);
                 }
                 if (u > 0) mbar_wait(bar(B_EMPTY + s), (u - 1) & 1, abort_flag, p.dev_status);
-                const uint32_t dst = base + p.off_stage + s * STAGE;
-                mbar_expect_tx(bar(B_FULL + s), STAGE);
+                const uint32_t dst = base + p.off_stage + s * TILE;
+                mbar_expect_tx(bar(B_FULL + s), TILE);
                 if (j >= TC) {   // active rows [128 x, 128 x + 128) of this kv head, fresh; rows past n_active read as zero
-                    const int x = j - TC;
-                    tma_load_5d(dst, &map_kn, 0, x * BK, 0, hk, b, bar(B_FULL + s));
-                    tma_load_5d(dst + TILE, &map_vn, 0, x * BK, 0, hk, b, bar(B_FULL + s));
+                    tma_load_5d(dst, (n & 1) ? &map_vn : &map_kn, 0, (j - TC) * BK, 0, hk, b, bar(B_FULL + s));
                 } else {
-                    const int key0 = (t_begin + j) * BK;
-                    tma_load_4d(dst, &map_k, 0, key0, 0, bh, bar(B_FULL + s));
-                    tma_load_4d(dst + TILE, &map_v, 0, key0, 0, bh, bar(B_FULL + s));
+                    tma_load_4d(dst, (n & 1) ? &map_v : &map_k, 0, (t_begin + j) * BK, 0, bh, bar(B_FULL + s));
                 }
             }
         }
@@ -335,9 +335,9 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             constexpr uint32_t IDESC_PV = instr_desc2(N, 1, 1);   // A = V tile (MN-major: d contiguous), B = P^T (MN-major)
             constexpr uint32_t QHALF = N * 128;                   // bytes of one 64-column half of the Q tile
             auto issue_s = [&](int j) {
-                const int s = j % NS;
+                const int s = (2 * j) % NS;
                 fence_after();
-                const uint32_t kst = base + p.off_stage + s * STAGE;
+                const uint32_t kst = base + p.off_stage + s * TILE;
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t koff = (k & 3) * 32;
@@ -345,6 +345,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                            smem_desc(base + (k >> 2) * QHALF + koff, 16, 1024), IDESC_S, k > 0);
                 }
                 commit(bar(B_SFULL + (j & 1)));
+                commit(bar(B_EMPTY + s));   // the K slot is free once these products have run
             };
             // S of tile j needs the tile (and its patch); P V of tile j needs P^T from the softmax.  Whichever is ready
             // is issued: P V of a tile does not wait for the next tile to land (its commit frees the stage for the
@@ -354,21 +355,22 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
             SpinGuard guard;
             while (next_pv < T) {
                 bool progressed = false;
-                if (next_s < T && next_s <= next_pv + 1 && mbar_try(bar(B_FULL + next_s % NS), (next_s / NS) & 1)) {
+                if (next_s < T && next_s <= next_pv + 1 && mbar_try(bar(B_FULL + (2 * next_s) % NS), ((2 * next_s) / NS) & 1)) {
                     issue_s(next_s);   // (the tile has landed)
                     ++next_s;
                     progressed = true;
                 }
-                if (mbar_try(bar(B_PFULL), next_pv & 1)) {
+                if (mbar_try(bar(B_PFULL), next_pv & 1) &&
+                    mbar_try(bar(B_FULL + (2 * next_pv + 1) % NS), ((2 * next_pv + 1) / NS) & 1)) {   // P^T is there, V has landed
                     const int j = next_pv;
-                    const uint32_t vst = base + p.off_stage + (j % NS) * STAGE + TILE;
+                    const uint32_t vst = base + p.off_stage + ((2 * j + 1) % NS) * TILE;
                     fence_after();
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
                         mma_ss(tmem + TM_O, smem_desc(vst + k * 2048, SUB, 1024), smem_desc(base + p.off_p + k * 2048, SUB, 1024),
                                IDESC_PV, (j > 0 || k > 0));
                     commit(bar(B_PVDONE));
-                    commit(bar(B_EMPTY + j % NS));
+                    commit(bar(B_EMPTY + (2 * j + 1) % NS));
                     ++next_pv;
                     progressed = true;
                 }
@@ -396,8 +398,10 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                 // thread reports after it has read its pieces.  (One TMA store per row and half took 3.5 us for 34
                 // rows: 136 requests of 128 bytes, served one after the other.)
                 const int x = j - TC;
-                mbar_wait(bar(B_FULL + j % NS), (j / NS) & 1, abort_flag, p.dev_status);   // the fresh tile has landed
-                const unsigned char* tile = gbase + p.off_stage + (j % NS) * STAGE;
+                mbar_wait(bar(B_FULL + (2 * j) % NS), ((2 * j) / NS) & 1, abort_flag, p.dev_status);           // the fresh K tile
+                mbar_wait(bar(B_FULL + (2 * j + 1) % NS), ((2 * j + 1) / NS) & 1, abort_flag, p.dev_status);   // and V tile
+                const unsigned char* ktile = gbase + p.off_stage + ((2 * j) % NS) * TILE;
+                const unsigned char* vtile = gbase + p.off_stage + ((2 * j + 1) % NS) * TILE;
                 const int ch = atid & 15;   // piece of the row: columns [8 ch, 8 ch + 8)
                 const int n_rows = min(BK, p.n_active - x * BK);
                 for (int r = atid >> 4; r < n_rows; r += kAuxThreads / 16) {
@@ -406,8 +410,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
                     if (pos < 0 || pos >= p.ctx_len) continue;
                     const uint32_t off = (ch >> 3) * SUB + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4);
                     const long long dst = (((long long)bh * p.ctx_len + pos) * HD + ch * 8);
-                    *reinterpret_cast<uint4*>(p.k_cache + dst) = *reinterpret_cast<const uint4*>(tile + off);
-                    *reinterpret_cast<uint4*>(p.v_cache + dst) = *reinterpret_cast<const uint4*>(tile + TILE + off);
+                    *reinterpret_cast<uint4*>(p.k_cache + dst) = *reinterpret_cast<const uint4*>(ktile + off);
+                    *reinterpret_cast<uint4*>(p.v_cache + dst) = *reinterpret_cast<const uint4*>(vtile + off);
                 }
             }
             // P^T of tile j is in shared memory
@@ -742,7 +746,7 @@ void carve(KeysPlan& pl, int n_active, int ns, bool fresh) {
     pl.off_p = off;
     off += (uint32_t)((pl.n_slots + 63) / 64) * SUB;
     pl.off_stage = off;
-    off += (uint32_t)ns * STAGE;
+    off += (uint32_t)ns * TILE;
     pl.off_list = off;
     off += fresh ? (uint32_t)n_active * 16u : 0u;
     pl.off_bar = off;
@@ -840,10 +844,10 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active, bool fresh) {
             const int visits = own ? (tps > pl.n_extra ? tps : pl.n_extra)
                                    : (tps > last_tiles + pl.n_extra ? tps : last_tiles + pl.n_extra);
             KeysPlan t = pl;
-            int ns = visits < kMaxStages ? visits : kMaxStages;
+            int ns = 2 * visits < kMaxStages ? 2 * visits : kMaxStages;   // ring slots: a K and a V slot per tile in flight
             carve(t, n_active, ns, fresh);
-            while (ns > 1 && t.smem_bytes > kSmemMax) carve(t, n_active, --ns, fresh);
-            if (t.smem_bytes > kSmemMax || (ns < 2 && visits > 1)) continue;
+            while (ns > 2 && t.smem_bytes > kSmemMax) carve(t, n_active, --ns, fresh);
+            if (t.smem_bytes > kSmemMax || (ns < 4 && visits > 1)) continue;
             // the exchange areas of the merge (2 c chunks) reuse the Q / P^T / stage memory
             if (c > 1 && 2 * (size_t)c * (pl.n_slots * dl + 2 * pl.n_slots) * 4 > t.off_list) continue;
             const int per_sm = (t.smem_bytes <= kSmemTwoPerSm && tm_cols <= 256) ? 2 : 1;
@@ -948,7 +952,7 @@ bool attend_skip_keys_supported(const ec_attn_desc& d, int n_active, bool fresh)
 
 void attend_skip_keys_describe(const ec_attn_desc& d, int n_active, bool fresh, char* buf, size_t len) {
     const KeysPlan pl = make_keys_plan(d, n_active, fresh);
-    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d stages=%d smem=%u ctas_per_sm=%d fresh_tiles=%d",
+    snprintf(buf, len, "attend_skip_keys_kernel<%d> grid=(%d,%d) cluster=%d ring_slots=%d smem=%u ctas_per_sm=%d fresh_tiles=%d",
              pl.n_slots, pl.n_splits, d.batch * d.n_kv_heads * pl.n_sub, pl.n_splits, pl.n_stages, pl.smem_bytes, pl.ctas_per_sm,
              pl.n_extra);
 }
