@@ -61,7 +61,9 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 128, HD = 128;
-constexpr int kAuxThreads = 64;           // two warps: cache update and row sums
+// auxiliary warps (cache update and row sums): two, or four for the 96-slot instantiation, whose row sums over twice
+// the columns otherwise trail the softmax and hold up the merge
+__host__ __device__ constexpr int aux_threads(int n) { return n > 64 ? 128 : 64; }
 constexpr uint32_t SUB = 128 * 128;        // [128 rows x 64 bf16], 128-byte swizzle: 16 KB
 constexpr uint32_t TILE = 2 * SUB;         // [128 x 128] bf16
 constexpr uint32_t STAGE = 2 * TILE;       // K tile + V tile: 64 KB
@@ -154,7 +156,7 @@ struct alignas(16) KeysShared {
 };
 
 template <int N>
-__global__ void __launch_bounds__(64 + (N > 64 ? 256 : 128) + kAuxThreads, N <= 64 ? 2 : 1)
+__global__ void __launch_bounds__(64 + (N > 64 ? 256 : 128) + aux_threads(N), N <= 64 ? 2 : 1)
 attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kn,
                         const __grid_constant__ CUtensorMap map_vn, const KeysParams p) {
@@ -162,6 +164,7 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     constexpr int WG = N > 64 ? 2 : 1;          // softmax warpgroups: each takes NH of a key's N scores
     constexpr int NH = N / WG;
     constexpr int kSoft = 128 * WG;
+    constexpr int kAuxThreads = aux_threads(N);
     constexpr int kThreads = 64 + kSoft + kAuxThreads;
     // tensor-memory columns: S^T x 2 and O^T at multiples of NP (the slots rounded up to 64 or 128)
     constexpr uint32_t NP = N <= 64 ? 64 : 128;
@@ -648,8 +651,38 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         const float* recv = reinterpret_cast<const float*>(gbase + recv_off);
         // a thread owns two adjacent output columns of a query row (one 4-byte store) and works out the row's weights
         // 2^(m_s - m) / l itself: the sixteen or so threads of a row repeat that, but nobody waits for a table
-        const int half_dl = min(DL, HD - split * DL) / 2;
-        if (!*abort_flag) {
+        const int own_dl = min(DL, HD - split * DL);   // output columns this CTA owns (even)
+        if (!*abort_flag && (DL & 3) == 0 && (own_dl & 3) == 0) {
+            // four adjacent output columns of a query row per item (one 8-byte store)
+            const int quads = own_dl / 4;
+            for (int idx = tid; idx < rows_total * quads; idx += kThreads) {
+                const int qq = idx / quads, dq = idx % quads;
+                float m = -INFINITY;
+#pragma unroll
+                for (int s = 0; s < 8; ++s)
+                    if (s < C) m = fmaxf(m, recv[s * chunk_floats + N * DL + qq]);
+                float l = 0.f;
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    if (s < C) {
+                        const float* ch = recv + s * chunk_floats;
+                        const float e = fast_exp2(ch[N * DL + qq] - m);
+                        const float4 v = *reinterpret_cast<const float4*>(ch + qq * DL + 4 * dq);
+                        l = fmaf(e, ch[N * DL + N + qq], l);
+                        a.x = fmaf(e, v.x, a.x);
+                        a.y = fmaf(e, v.y, a.y);
+                        a.z = fmaf(e, v.z, a.z);
+                        a.w = fmaf(e, v.w, a.w);
+                    }
+                }
+                const float inv = 1.f / l;
+                const int i = i0 + qq / p.group, jh = qq % p.group;
+                __nv_bfloat16* dst = p.out + (((long long)b * p.n_active + i) * p.n_q_heads + hq0 + jh) * HD + split * DL + 4 * dq;
+                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(a.x * inv, a.y * inv), pack_bf16x2(a.z * inv, a.w * inv));
+            }
+        } else if (!*abort_flag) {
+            const int half_dl = own_dl / 2;
             for (int idx = tid; idx < rows_total * half_dl; idx += kThreads) {
                 const int qq = idx / half_dl, dp = idx % half_dl;
                 float ms[8], ls[8];
@@ -771,7 +804,7 @@ int resident_clusters_of(int c, uint32_t smem) {
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(c, 1, 1);
-    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + kAuxThreads, 1, 1);
+    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + aux_threads(N), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -922,7 +955,7 @@ cudaError_t launch_n(const KeysPlan& pl, const KeysParams& p, const CUtensorMap&
         return ea;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(pl.n_splits, bh, 1);
-    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + kAuxThreads, 1, 1);
+    cfg.blockDim = dim3(64 + (N > 64 ? 256 : 128) + aux_threads(N), 1, 1);
     cfg.dynamicSmemBytes = pl.smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];
