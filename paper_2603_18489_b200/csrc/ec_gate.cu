@@ -6,7 +6,8 @@
 // R*V*sizeof(elem) bytes are read exactly once; the arithmetic is about seven instructions per element.
 //   grid  = (splits, R): CTA (s, r) owns the columns [s*chunk, (s+1)*chunk) of row r; the split count is
 //           chosen so that the whole grid is about one resident wave (4 CTAs per SM);
-//   CTA   : 8 consumer warps and one producer warp.  The producer's lane 0 moves the chunk through a ring of
+//   CTA   : (inputs below 24 MB; larger ones: every thread loads its own vectors through four rolling registers,
+//           no producer warp)  8 consumer warps and one producer warp.  The producer's lane 0 moves the chunk through a ring of
 //           three 16 KB stages in shared memory with bulk copies (cp.async.bulk, completion on an mbarrier, L2
 //           evict-first), as far ahead as the ring allows, so the bytes in flight per SM are the rings of its
 //           resident CTAs and do not depend on the consumers' registers;
@@ -47,6 +48,7 @@ constexpr int kVec = 8;  // columns per thread in one slab of kGateThreads * kVe
 constexpr int kMaxSplits = 96;
 constexpr float kDClamp = -150.0f;  // 2^-150 flushes to 0 (ftz)
 constexpr int kStages = 3;                          // ring of staged buffers per CTA
+constexpr int kInFlight = 4;                        // rolling variant: 16-byte vectors a thread keeps in flight
 constexpr int kStageVecs = 4 * kGateThreads;        // 16-byte vectors per stage: four per consumer thread
 constexpr uint32_t kStageBytes = kStageVecs * 16u;
 constexpr int kPoison = 1 << 20;                    // added to a ticket by a CTA whose wait gave up
@@ -249,8 +251,12 @@ __device__ __forceinline__ float finish_row(const GateParams& p, int row, int la
     return H;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kGateThreads + 32, kCtasPerSm) gate_kernel(const GateParams p) {
+// kStaged: the logits come through the bulk-copy ring (a producer warp on top of the consumers); otherwise every
+// thread loads its own vectors into a rolling set of kInFlight registers.  The ring wins on small inputs (three
+// stages are on their way before any consumer has started: 7.5 against 8.3 us at [32, 126464]), the rolling loads on
+// large ones (17.8 against 19.7 us at [256, 126464]): the host picks by size.
+template <typename T, bool kStaged>
+__global__ void __launch_bounds__(kGateThreads + (kStaged ? 32 : 0), kCtasPerSm) gate_kernel(const GateParams p) {
     __shared__ float s_m[kGateThreads / 32];
     __shared__ int s_i[kGateThreads / 32];
     __shared__ float s_S[kGateThreads / 32], s_T[kGateThreads / 32];
@@ -301,16 +307,18 @@ __global__ void __launch_bounds__(kGateThreads + 32, kCtasPerSm) gate_kernel(con
     const int n_vec = (c_end - c0) / EPV;                                  // whole vectors of the chunk
     const int n_stage = (n_vec + kStageVecs - 1) / kStageVecs;
     if (tid == 0) {
+        if (kStaged) {
 #pragma unroll
-        for (int i = 0; i < kStages; ++i) { tc::mbar_init(full0 + 8u * i, 1); tc::mbar_init(empty0 + 8u * i, kGateThreads / 32); }
+            for (int i = 0; i < kStages; ++i) { tc::mbar_init(full0 + 8u * i, 1); tc::mbar_init(empty0 + 8u * i, kGateThreads / 32); }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
         s_abort = 0;
         s_issued = -1;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     pdl_wait();                 // the previous kernel of the stream has completed: the logits are final
     pdl_launch_dependents();
-    if (warp == kGateThreads / 32) {            // the producer warp
+    if (kStaged && warp == kGateThreads / 32) {            // the producer warp
         if (lane == 0) {
             const unsigned char* src = reinterpret_cast<const unsigned char*>(rowp + c0);
             const uint64_t policy = evict_first_policy();
@@ -348,7 +356,30 @@ __global__ void __launch_bounds__(kGateThreads + 32, kCtasPerSm) gate_kernel(con
             T2 = fma2(e2, d2, T2);
         }
     };
-    for (int s = 0; s < n_stage; ++s) {
+    if (!kStaged) {
+        // Thread t owns the vectors t, t + 256, ... of the chunk.  They pass through a rolling set of kInFlight
+        // registers: as soon as a vector has been consumed its register is given to the load kInFlight vectors ahead.
+        constexpr int kVStride = kGateThreads * EPV;
+        const int n_mine = n_vec > tid ? (n_vec - tid + kGateThreads - 1) / kGateThreads : 0;
+        const T* mine = rowp + c0 + tid * EPV;
+        uint4 raw[kInFlight];
+#pragma unroll
+        for (int v = 0; v < kInFlight; ++v)
+            if (v < n_mine) raw[v] = __ldcs(reinterpret_cast<const uint4*>(mine + (long long)v * kVStride));   // streamed once
+        int i0 = 0;
+        for (; i0 + kInFlight <= n_mine; i0 += kInFlight) {
+#pragma unroll
+            for (int v = 0; v < kInFlight; ++v) {
+                consume(raw[v], c0 + (i0 + v) * kVStride + tid * EPV);
+                if (i0 + v + kInFlight < n_mine)
+                    raw[v] = __ldcs(reinterpret_cast<const uint4*>(mine + (long long)(i0 + v + kInFlight) * kVStride));
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < kInFlight; ++v)
+            if (i0 + v < n_mine) consume(raw[v], c0 + (i0 + v) * kVStride + tid * EPV);
+    }
+    for (int s = 0; kStaged && s < n_stage; ++s) {
         const int slot = s % kStages;
         tc::mbar_wait(full0 + 8u * slot, (s / kStages) & 1, &s_abort, nullptr);
         if (s_abort) break;
@@ -649,22 +680,24 @@ void plan_chunks(int n_rows, int vocab, int* splits, int* chunk, int max_splits 
     *splits = (int)((vocab + per - 1) / per);
 }
 
-template <typename T>
+template <typename T, bool kStaged>
 cudaError_t launch_t(const GateParams& p, cudaStream_t stream) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(p.splits, p.n_rows, 1);
-    cfg.blockDim = dim3(kGateThreads + 32, 1, 1);    // the consumer warps and the producer warp
-    cfg.dynamicSmemBytes = kStages * kStageBytes;
-    static PerDeviceOnce once;
-    const cudaError_t e = ensure_dynamic_smem(once, gate_kernel<T>, kStages * kStageBytes);
-    if (e != cudaSuccess) return e;
+    cfg.blockDim = dim3(kGateThreads + (kStaged ? 32 : 0), 1, 1);    // the consumer warps (and the producer warp)
+    cfg.dynamicSmemBytes = kStaged ? kStages * kStageBytes : 0;
+    if (kStaged) {
+        static PerDeviceOnce once;
+        const cudaError_t e = ensure_dynamic_smem(once, gate_kernel<T, kStaged>, kStages * kStageBytes);
+        if (e != cudaSuccess) return e;
+    }
     cfg.stream = stream;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // launch latency may overlap the previous kernel's tail
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gate_kernel<T>, p);
+    return cudaLaunchKernelEx(&cfg, gate_kernel<T, kStaged>, p);
 }
 
 }  // namespace
@@ -711,7 +744,12 @@ cudaError_t launch_gate(const GateArgs& a, cudaStream_t stream) {
     if (p.splits > kMaxSplits) return cudaErrorInvalidValue;   // vocab > 96 * 8192: rejected by the API layer before this
     p.single_level = (a.rows_per_seq <= kSingleLevelMaxRows && p.splits <= 32) ? 1 : 0;
     if (one_cta_finish && !p.single_level) return cudaErrorInvalidValue;   // rows_per_seq > 64 or vocab > 32 * 8192 * ...: rejected by the API layer
-    return a.dtype == EC_BF16 ? launch_t<__nv_bfloat16>(p, stream) : launch_t<float>(p, stream);
+    // small inputs through the bulk-copy ring, large ones (more than a few chunks per CTA slot) with per-thread loads
+    const size_t bytes = (size_t)a.n_rows * a.vocab * (a.dtype == EC_BF16 ? 2 : 4);
+    const bool staged = bytes < ((size_t)24 << 20);
+    if (a.dtype == EC_BF16)
+        return staged ? launch_t<__nv_bfloat16, true>(p, stream) : launch_t<__nv_bfloat16, false>(p, stream);
+    return staged ? launch_t<float, true>(p, stream) : launch_t<float, false>(p, stream);
 }
 
 }  // namespace ec

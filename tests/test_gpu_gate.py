@@ -156,3 +156,18 @@ def test_the_three_candidate_metrics(name, R, rps):
     fin = np.isfinite(m["max_conf"])
     assert np.array_equal(np.isfinite(g["max_conf"]), fin) and not fin[0] and g["entropy_sum"][0] == 0.0
     assert np.all(np.abs(g["max_conf"][fin].astype(np.float64) - m["max_conf"][fin]) <= 1e-5 * m["max_conf"][fin])
+
+
+@pytest.mark.parametrize("dtype,R,V,stride,rps", [(syn.F32, 96, 126464, 126464, 32), (syn.BF16, 200, 126466, 126472, 40),
+                                                  (syn.F32, 48, 152064, 152064, 48)])
+def test_gate_on_inputs_large_enough_for_the_per_thread_loads(dtype, R, V, stride, rps):
+    """From 24 MB of logits on, the gate's threads load their own vectors (rolling registers) instead of reading a
+    bulk-copy ring: both storage types, a padded stride with a ragged vocabulary, sequences of 40 and 48 rows (the
+    benchmark shape [256, 126464] bf16 is covered by test_gate_on_benchmark_shapes)."""
+    assert R * V * (4 if dtype == syn.F32 else 2) >= 24 << 20
+    st = syn.logits_rows(R, V, dtype, cfg_id=8, row_stride=stride)
+    flags = syn.decoded_flags(R, 7, rps, cfg_id=8)
+    tau = 2.0
+    g = _run_gpu(st["logits"], dtype, V, flags, tau, rps)
+    o = oracle.entropy_gate(st["logits"], dtype, V, flags, tau, rps)
+    _compare(g, o, tau)
