@@ -55,8 +55,8 @@ K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dr
 NCU_TRAFFIC = {
     "attend_skip": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-         "sha256": "56358dbda13ef444eae93ef1111ad7fa45d20efc64d2a78e4774ac8a6b877f89",
-         "bytes_per_launch": {"c2_llada_l768": 13500000, "c5_llada_l4096": 68670000}},
+         "sha256": "ef2b91e7c5b647875f56f086e856d71bed9863a7420a5b46571e0b2b939e7265",
+         "bytes_per_launch": {"c2_llada_l768": 13510000, "c5_llada_l4096": 68760000}},
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
          "sha256": "bfec166c49fcaea673858dc2e86bfa2b1bffe4d191e2c41857dac13d2d180d5a",
          "bytes_per_launch": {"c5_llada_l4096_b8": 552480000}}],
@@ -66,8 +66,8 @@ NCU_TRAFFIC = {
          "bytes_per_launch": {"c2_llada_l768": 18930000, "c4_llada_l2048": 62770000, "c5_llada_l4096": 176240000}}],
     "entropy_gate": [
         {"source": "paper_2603_18489_b200/csrc/ec_gate.cu",
-         "sha256": "9aff17035d14500e5378489b0f9cb64e1b4f42fbe658d39056e2c7edeb701d42",
-         "bytes_per_launch": {"c5_llada_l4096": 8140000, "c5_llada_l4096_b8": 65130000}}],
+         "sha256": "519bc6a99b3932ab141af3aa77056dff693970d2254c54c7a023263874293215",
+         "bytes_per_launch": {"c5_llada_l4096": 8140000, "c5_llada_l4096_b8": 65060000}}],
 }
 
 
