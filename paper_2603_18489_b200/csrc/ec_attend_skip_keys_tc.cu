@@ -126,6 +126,8 @@ struct KeysParams {
     int n_sub_r;      // row chunks = ceil(n_active / rows_chunk)
     int n_sub;        // CTA columns per kv head = ((H_q / H_kv) / group) * n_sub_r
     int n_splits, tiles_per_split, n_stages;
+    int shift;        // 1: the first CTA of the cluster takes one cache tile more and the last, which also visits the
+                      // fresh tiles, one less (ranges of the CTAs in between move up by one tile)
     int n_extra;      // key tiles of fresh rows attended by the last CTA of every cluster (0: nothing to refresh)
     int dl;           // output columns merged by one CTA of the cluster (even; the last CTA may own fewer)
     int q_tma;        // 1: the producer fetches Q with one TMA box (one query head per column); 0: softmax warps stage it
@@ -190,8 +192,8 @@ attend_skip_keys_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     const int C = p.n_splits;
     const int DL = p.dl;
     const int n_tiles_total = (p.ctx_len + BK - 1) / BK;
-    const int t_begin = split * p.tiles_per_split;
-    const int t_end = min(n_tiles_total, t_begin + p.tiles_per_split);
+    const int t_begin = split * p.tiles_per_split + (split > 0 ? p.shift : 0);
+    const int t_end = min(n_tiles_total, (split + 1) * p.tiles_per_split + p.shift);
     const int TC = max(0, t_end - t_begin);                  // cache tiles of this CTA
     const int NS = p.n_stages;       // ring slots: tile j has K in slot 2j mod NS and V in slot (2j + 1) mod NS
     const bool refresh = p.k_new != nullptr;
@@ -761,7 +763,7 @@ bool make_q_map(CUtensorMap* map, const void* q, int batch, int n_active, int n_
 struct KeysPlan {
     bool ok;
     int group, rows_chunk, n_sub_r, n_sub;   // heads and active rows per CTA column, row chunks, CTA columns per kv head
-    int n_slots, n_splits, tiles_per_split, n_stages, n_extra, dl, ctas_per_sm;
+    int n_slots, n_splits, tiles_per_split, n_stages, n_extra, dl, ctas_per_sm, shift;
     uint32_t off_p, off_stage, off_list, off_bar, smem_bytes;
 };
 
@@ -896,6 +898,10 @@ KeysPlan make_keys_plan(const ec_attn_desc& d, int n_active, bool fresh) {
                 best_ctas = ctas;
                 pl.n_splits = c;
                 pl.tiles_per_split = tps;
+                // The CTA that also visits the fresh tiles has one visit more than its peers, and the cluster waits for
+                // it at the merge.  The memory system serves whoever asks, so giving that CTA one cache tile less (and
+                // the first CTA one more) lets it finish its stream early and spend the difference on the extra visit.
+                pl.shift = (fresh && !own && cs >= 2 && tps >= 2 && last_tiles == tps) ? 1 : 0;
                 pl.dl = dl;
                 pl.ctas_per_sm = per_sm;
                 pl.n_stages = ns;
@@ -1024,6 +1030,7 @@ cudaError_t launch_attend_skip_keys(const AttendArgs& a, const void* k_new, cons
     p.n_sub = pl.n_sub;
     p.n_splits = pl.n_splits;
     p.tiles_per_split = pl.tiles_per_split;
+    p.shift = pl.shift;
     p.n_stages = pl.n_stages;
     p.n_extra = pl.n_extra;
     p.dl = pl.dl;
