@@ -55,8 +55,8 @@ K64_WORKLOADS = ("c4_llada_l2048", "c5_llada_l4096", "c5_llada_l4096_b8", "c5_dr
 NCU_TRAFFIC = {
     "attend_skip": [
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_keys_tc.cu",
-         "sha256": "ef2b91e7c5b647875f56f086e856d71bed9863a7420a5b46571e0b2b939e7265",
-         "bytes_per_launch": {"c2_llada_l768": 13510000, "c5_llada_l4096": 68760000}},
+         "sha256": "55eea1c65c1cfe60b79f17c4d0f5c2d222cf29ddff308fb432c5a73e07d8b972",
+         "bytes_per_launch": {"c2_llada_l768": 13400000, "c5_llada_l4096": 68730000}},
         {"source": "paper_2603_18489_b200/csrc/ec_attend_skip_tc.cu",
          "sha256": "bfec166c49fcaea673858dc2e86bfa2b1bffe4d191e2c41857dac13d2d180d5a",
          "bytes_per_launch": {"c5_llada_l4096_b8": 552480000}}],
