@@ -268,3 +268,56 @@ def test_recompute_step_whose_last_wave_is_cut_along_the_keys(name, Hq, Hkv, L, 
     rows = sorted(set(rng.choice(L, 10, replace=False).tolist() + rng.choice(np.arange(L // 2, L), 14, replace=False).tolist()
                       + [0, L - 1]))
     _check(w, t, row_sel=rows)
+
+
+def test_cut_last_wave_with_an_explicit_permuted_index_list():
+    """Every row active but given as a shuffled index list: the refresh runs as its own launch, then the dense kernel
+    with its last wave cut along the keys and the combine launch; output rows follow the list's order."""
+    import paper_2603_18489_b200 as ec
+
+    L, Hq, Hkv = 2048, 19, 19
+    w = syn.Workload(96, "h19_l2048_perm", syn.BF16, 1, Hq, Hkv, 128, L - 256, 256, 32, 2, 1024)
+    d = ec.make_desc(1, L, Hq, Hkv, 128, syn.BF16)
+    got = ec.ec_attend_kernel_name(d, L, True, True)
+    assert "refresh_kernel" in got and "attend_dense_kernel" in got and "cut_units=4x4" in got, got
+    idx = syn.arbitrary_active_idx(1, L, L, seed=5)
+    t = syn.attn_inputs(w, L, active_idx=idx, std_qk=0.35, salt=4)
+    rows = sorted(set(np.random.Generator(np.random.PCG64(9)).choice(L, 20, replace=False).tolist() + [0, L - 1]))
+    _check(w, t, row_sel=rows)
+
+
+def test_back_to_back_layers_with_the_flag_at_the_papers_default_budget():
+    """The same unsynchronised passes as above with k = 64 (96 active rows): the 96-slot instantiation with its
+    five-slot ring and four auxiliary warps."""
+    import dataclasses
+
+    import paper_2603_18489_b200 as ec
+
+    w = dataclasses.replace(syn.WORKLOADS["c4_llada_l2048"], k_recent=64)
+    n, n_layers, n_pass = w.n_skip_rows, 3, 2
+    d = ec.make_desc(w.batch, w.ctx_len, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, flags=ec.EC_ATTN_CACHE_SETTLED)
+    assert ec.ec_attend_kernel_name(d, n, True, True).startswith("attend_skip_keys_kernel<96>")
+    ins = [[syn.attn_inputs(w, n, step=p, salt=70 + l, block_no=p) for l in range(n_layers)] for p in range(n_pass)]
+    kc = [ins[0][l]["k_cache"].copy() for l in range(n_layers)]
+    vc = [ins[0][l]["v_cache"].copy() for l in range(n_layers)]
+    gk, gv = [to_dev(a) for a in kc], [to_dev(a) for a in vc]
+    dev = [[{k: to_dev(ins[p][l][k]) for k in ("q", "k_new", "v_new", "active_idx")} for l in range(n_layers)]
+           for p in range(n_pass)]
+    outs = [[torch.empty_like(dev[p][l]["q"]) for l in range(n_layers)] for p in range(n_pass)]
+    ws = ec.new_workspace(max(16, ec.ec_attend_workspace_bytes(d, n)))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    for p in range(n_pass):
+        for l in range(n_layers):
+            t = dev[p][l]
+            ec.ec_attend(d, t["q"], t["k_new"], t["v_new"], gk[l], gv[l], t["active_idx"], out=outs[p][l],
+                         workspace=ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for p in range(n_pass):
+        for l in range(n_layers):
+            t = ins[p][l]
+            ref = oracle.refresh_and_attend(t["q"], t["k_new"], t["v_new"], kc[l], vc[l], t["active_idx"], w.dtype)
+            assert np.abs(to_f64(outs[p][l]) - ref).max() <= BF16_TOL, (p, l)
+    for l in range(n_layers):
+        assert np.array_equal(to_storage(gk[l]), kc[l]) and np.array_equal(to_storage(gv[l]), vc[l])
